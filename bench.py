@@ -1,0 +1,434 @@
+#!/usr/bin/env python
+"""Benchmark of the weighted aggregate + update path.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
+
+One step = one pass of the synchronous hot path on the ResNet-50-shaped mixed-precision
+workload (K=16 workers, 25.6M parameters, bfloat16 gradients, float32 master parameters and
+momentum, 25 MiB buckets): a controller re-batch from freshly jittered throughputs (host), the
+batch-size weights, the fused K-way weighted sum + momentum update + squared norm (one kernel
+launch over all buckets).  The asynchronous arrival path and the other configurations are timed
+in the same run and reported under "extras".  Prints ONE JSON line on rank 0.
+
+Multi-GPU: the path has no exchange step, so N GPUs run N independent replicas; the value is
+the parameters all replicas updated divided by the slowest replica's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+HEADLINE = "resnet50_bf16"
+METRIC = "params/sec, weighted aggregate+update (achieved HBM GB/s in roofline)"
+UNIT = "params/s"
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Reads SM clock and clock-event reasons of one GPU every 20 ms while the timed region runs."""
+
+    REASONS = {
+        0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+        0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def visible_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# --------------------------------------------------------------------------------------------
+# helpers
+# --------------------------------------------------------------------------------------------
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    for f in ("kernels.cuh", "omni.cu"):
+        h.update((ROOT / "paper_2503_17469_b200" / "csrc" / f).read_bytes())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(name: str):
+    """DRAM bytes per launch from the committed ncu capture, or None when the kernel source has
+    changed since the counters were taken."""
+    p = ROOT / "profiles" / "traffic.json"
+    if not p.exists():
+        return None
+    try:
+        rec = json.loads(p.read_text()).get(name)
+        if rec and rec.get("kernel_source_hash") == kernel_source_hash():
+            return rec["dram_bytes_per_launch"]
+    except Exception:
+        pass
+    return None
+
+
+def throughput_schedule(cfg, n, W, torch):
+    gen = torch.Generator().manual_seed(cfg.seed)
+    base = list(cfg.throughputs) if cfg.throughputs else W.draw_throughputs(cfg.K, gen, cfg.ratio)
+    return base, [W.jitter_throughputs(base, gen) for _ in range(n)]
+
+
+class BspJob:
+    """Buffers + context of one synchronous configuration on the current device."""
+
+    def __init__(self, name, torch, W, B, with_lp=False):
+        self.cfg = cfg = W.config(name)
+        self.torch = torch
+        self.buf = W.make_buffers(cfg, torch.device("cuda", torch.cuda.current_device()))
+        lay = self.buf.layout
+        self.theta_lp = torch.zeros(lay.total, dtype=torch.bfloat16, device=self.buf.theta.device) if with_lp else None
+        self.omni = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.BSP)
+        self.buckets = B.BucketSet.from_flat(lay, self.buf.theta, self.buf.grads, self.buf.v, self.theta_lp)
+        self.bytes_per_step = cfg.bytes_per_param(with_lp) * cfg.P
+        self.W = W
+
+    def run(self, steps, schedule):
+        o, bs, cfg = self.omni, self.buckets, self.cfg
+        for i in range(steps):
+            b, _ = o.rebatch(schedule[i % len(schedule)])
+            o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+
+    def timed(self, steps, warmup, schedule, sampler=None, barrier=None):
+        torch = self.torch
+        self.run(warmup, schedule)
+        torch.cuda.synchronize()
+        if barrier:
+            barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = self.omni.kernel_launches
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.__enter__()
+        e0.record()
+        self.run(steps, schedule)
+        e1.record()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.__exit__()
+        if barrier:
+            barrier()
+        return e0.elapsed_time(e1), self.omni.kernel_launches - l0
+
+
+def bsp_line(job, ms, steps, launches, peak):
+    per_launch_s = ms * 1e-3 / max(launches, 1)
+    gbs = job.bytes_per_step * steps / max(launches, 1) / per_launch_s / 1e9
+    return {"params_per_s": job.cfg.P * steps / (ms * 1e-3), "ms_per_step": ms / steps, "achieved_gbs": gbs,
+            "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+            "bytes_per_param": job.bytes_per_step // job.cfg.P, "launches_per_step": launches / steps}
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle legs
+# --------------------------------------------------------------------------------------------
+def oracle_sample(name, target_s, torch, W):
+    """Times the single-threaded oracle on a prefix of the configuration's first bucket."""
+    from oracle import oracle as O
+    import numpy as np
+
+    cfg = W.config(name)
+    n = min(cfg.layout().buckets[0].n, 4_000_000)
+    gen = torch.Generator().manual_seed(cfg.seed)
+    gdt = torch.bfloat16 if cfg.grad_dtype == "bf16" else torch.float32
+    g = []
+    for _ in range(cfg.K):
+        t = torch.empty(n).normal_(0, 1e-3, generator=gen).to(gdt)
+        g.append(t.view(torch.int16).numpy().view(np.uint16).copy() if gdt == torch.bfloat16 else t.numpy().copy())
+    theta = torch.empty(n).normal_(0, cfg.param_std, generator=gen).numpy().copy()
+    v = np.zeros(n, np.float32)
+    ctl = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha)
+    base, sched = throughput_schedule(cfg, 64, W, torch)
+
+    def step(i):
+        b, _ = ctl.rebatch(sched[i % len(sched)])
+        O.bsp_step_f32(g, b, theta, v, cfg.lr, cfg.momentum, cfg.weight_decay)
+
+    return n, step
+
+
+def cpu_baseline(name, target_s, torch, W):
+    n, step = oracle_sample(name, target_s, torch, W)
+    step(0)
+    t0 = time.perf_counter()
+    step(1)
+    one = time.perf_counter() - t0
+    reps = max(1, int(target_s / max(one, 1e-6)))
+    t0 = time.perf_counter()
+    for i in range(reps):
+        step(2 + i)
+    dt = time.perf_counter() - t0
+    return {"value": n * reps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{reps} steps over the first {n} elements of bucket 0 of {name} (K and dtypes as configured), "
+                      f"single thread, {dt:.1f} s",
+            "host_cores_available": len(os.sched_getaffinity(0))}
+
+
+def reference_arm(args, torch, W):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n, step = oracle_sample(HEADLINE, 0, torch, W)
+    cfg = W.config(HEADLINE)
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = (f"each step = controller re-batch + oracle step over the first {n} elements of bucket 0 of {HEADLINE}, "
+              f"single thread")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": HEADLINE, "K": cfg.K, "params": cfg.P, "grad_dtype": cfg.grad_dtype,
+                       "global_batch": cfg.global_batch, "sample_elements": n},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# main
+# --------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="omni", choices=["omni", "reference"])
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2503_17469_b200 import workloads as W
+
+    if args.impl == "reference":
+        reference_arm(args, torch, W)
+        return
+
+    from paper_2503_17469_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    B.lib()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if not dist:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peak, peak_kind = measured_peak()
+    job = BspJob(HEADLINE, torch, W, B)
+    cfg = job.cfg
+    _, sched = throughput_schedule(cfg, 256, W, torch)
+    sampler = ClockSampler(visible_index(local))
+    ms, launches = job.timed(args.steps, args.warmup, sched, sampler, barrier)
+    ms = max_over_ranks(ms)
+    line_main = bsp_line(job, ms, args.steps, launches, peak)
+    grid, block = job.omni.query_launch(cfg.K, B.BF16)
+
+    # end to end: gradients arrive in pinned host memory, every step copies them in and reads the norm back
+    e2e_steps = max(3, min(args.steps, 20))
+    host = [[g[bk.start:bk.start + bk.n].cpu().pin_memory() for g in job.buf.grads] for bk in job.buf.layout.buckets]
+    h2d = sum(t.numel() * t.element_size() for row in host for t in row)
+
+    def e2e_run(n):
+        for i in range(n):
+            b, _ = job.omni.rebatch(sched[i % len(sched)])
+            job.omni.aggregate_bsp_host(job.buckets, host, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+
+    e2e_run(3)
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    e2e_run(e2e_steps)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks(max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3))
+    del host
+
+    extras = {}
+    if rank == 0 and world == 1 and not args.no_extras:
+        extras = run_extras(torch, W, B, peak, job)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(HEADLINE, 12.0, torch, W)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": world * line_main["params_per_s"], "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": line_main["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": HEADLINE, "K": cfg.K, "params": cfg.P, "tensors": len(cfg.shapes),
+                       "buckets": len(job.buf.layout.buckets), "grad_dtype": "bf16", "master_dtype": "f32",
+                       "global_batch": cfg.global_batch, "lr": cfg.lr, "momentum": cfg.momentum,
+                       "rebatch": "every step", "l2": "inputs exceed L2 (1.23 GB touched per step)",
+                       "multi_gpu": "replicas only", "grid": grid, "block": block},
+            "achieved_hbm_gbs": line_main["achieved_gbs"],
+            "pct_of_nominal_8TBs": 100 * line_main["frac_of_nominal_8TBs"],
+            "roofline": {"bound": "hbm", "achieved": line_main["achieved_gbs"], "peak": peak, "unit": "GB/s",
+                         "frac": line_main["frac_of_measured"], "peak_source": f"of {peak_kind}",
+                         "kernel": "bsp_fused_kernel<bf16,16>", "bytes_per_launch": job.bytes_per_step,
+                         "traffic": recorded_traffic("bsp_fused_bf16_k16")},
+            "e2e": {"value": world * cfg.P * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": 8, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": launches,
+            "clocks": sampler.summary(),
+            "cpu_baseline": cpu,
+            "extras": extras,
+        }
+        print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_extras(torch, W, B, peak, headline_job):
+    """The other configurations, each timed with CUDA events after warm-up (not part of `value`)."""
+    out = {}
+    del headline_job
+    torch.cuda.empty_cache()
+    for name, steps, lp in (("resnet50_bf16", 500, True), ("resnet50_f32", 500, False), ("resnet18", 1000, False),
+                            ("vgg16", 40, False), ("tiny", 2000, False)):
+        job = BspJob(name, torch, W, B, with_lp=lp)
+        _, sched = throughput_schedule(job.cfg, 64, W, torch)
+        ms, launches = job.timed(steps, 5, sched)
+        key = name + ("+lp_copy" if lp else "")
+        out[key] = bsp_line(job, ms, steps, launches, peak)
+        if name == "tiny":
+            out[key]["note"] = "33.6 MB working set: L2-resident and launch-bound, not an HBM figure"
+        del job
+        torch.cuda.empty_cache()
+    # asynchronous arrivals: 1000 single-worker gradients with controller feedback
+    cfg = W.config("resnet50_asp")
+    buf = W.make_buffers(cfg, torch.device("cuda", torch.cuda.current_device()))
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.ASP)
+    bs = B.BucketSet.from_flat(buf.layout, buf.theta, buf.grads)
+    gen = torch.Generator().manual_seed(cfg.seed)
+    T = W.draw_throughputs(cfg.K, gen, cfg.ratio)
+    u = torch.rand(cfg.steps + 50, generator=gen, dtype=torch.float64).tolist()
+    b = [cfg.global_batch // cfg.K] * cfg.K
+    last = [0] * cfg.K
+
+    def arrivals(i0, n):
+        for i in range(i0, i0 + n):
+            k = W.pick_worker(u[i], [T[j] / b[j] for j in range(cfg.K)])
+            o.apply_asp(bs, k, b[k], i - last[k], cfg.lr)
+            last[k] = i + 1
+            b[k] = o.asp_report(k, b[k], T[k])
+
+    arrivals(0, 50)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = o.kernel_launches
+    e0.record()
+    arrivals(50, cfg.steps)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    st = o.stats()
+    gbs = cfg.bytes_per_param() * cfg.P * cfg.steps / (ms * 1e-3) / 1e9
+    out["resnet50_asp"] = {"params_per_s": cfg.P * cfg.steps / (ms * 1e-3), "ms_per_arrival": ms / cfg.steps,
+                           "achieved_gbs": gbs, "frac_of_measured": gbs / peak,
+                           "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_param": cfg.bytes_per_param(),
+                           "launches_per_arrival": (o.kernel_launches - l0) / cfg.steps, "tau_max": st.tau_max,
+                           "tau_hist_0_31_overflow": st.tau_hist}
+    return out
+
+
+if __name__ == "__main__":
+    main()

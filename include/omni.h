@@ -1,0 +1,181 @@
+/*
+ * omni.h -- C ABI of the OmniLearn data-parallel hot path on one GPU.
+ *
+ * The library implements, for K workers whose gradients sit in K device buffers:
+ *   - the proportional batch-size controller (paper Eq. 6a/6b, dead-band Eq. 7, batch bounds,
+ *     global-batch rule Eq. 8; procedures getBsz of Algorithm 1 and evalBsz of Algorithm 2),
+ *   - the batch-size-weighted aggregation of the K gradients fused with the parameter update
+ *     (Eq. 4b, Eq. 4c; Algorithm 1 "AllReduce(lambda_k g)" and "theta - eta gbar"),
+ *   - the asynchronous per-arrival update with the batch-scaled learning rate
+ *     (Eq. 5b; Algorithm 2 "eta_k = eta b / B", "theta - eta_k g").
+ *
+ * Conventions
+ *   - Every function returns 0 (OMNI_OK) or a negative omni_status.  Nothing throws, aborts or
+ *     traps.  Arguments are validated before any state changes or any kernel is enqueued: a
+ *     failed call leaves the context and all buffers as they were.
+ *   - "device pointer" = memory of the CUDA device that is current when the call is made;
+ *     "host pointer" = ordinary host memory.  Parameter-sized buffers are owned by the caller
+ *     and must stay alive until the stream has executed the call.
+ *   - Kernels are enqueued on the caller's stream (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and the call returns without synchronising, unless stated otherwise.
+ *   - A context is not thread-safe.  It owns a small device workspace (per-block partial sums
+ *     and the gradient-norm cell, a few tens of KB) that is allocated by the first call that
+ *     launches a kernel and freed by omni_destroy; calls on different streams that share a
+ *     context and overlap on the GPU race on it.
+ *   - OMNI_MAX_K = 32 workers.
+ */
+#ifndef OMNI_H_
+#define OMNI_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OMNI_MAX_K 32
+#define OMNI_TAU_BINS 33 /* staleness 0..31 and one overflow bin */
+
+typedef enum {
+    OMNI_OK = 0,
+    OMNI_ERR_NULL = -1,            /* a required pointer is NULL */
+    OMNI_ERR_BAD_K = -2,           /* K outside 1..OMNI_MAX_K */
+    OMNI_ERR_BAD_WORKER = -3,      /* worker index outside 0..K-1 */
+    OMNI_ERR_BAD_BATCH = -4,       /* some b_k < 1, or sum b_k != B in synchronous mode */
+    OMNI_ERR_INFEASIBLE = -5,      /* K*b_min > B or K*b_max < B in synchronous mode */
+    OMNI_ERR_BAD_MEASUREMENT = -6, /* throughput/time not finite or <= 0 */
+    OMNI_ERR_ALIGN = -7,           /* a device pointer is not 16-byte aligned */
+    OMNI_ERR_BAD_TAU = -8,         /* negative staleness */
+    OMNI_ERR_CUDA = -9,            /* a CUDA call failed; see omni_last_cuda_error */
+    OMNI_ERR_TIMEOUT = -10,        /* a bounded device-side wait ran out */
+    OMNI_ERR_BAD_CONFIG = -11,     /* invalid omni_config field or call argument */
+    OMNI_ERR_TOO_LARGE = -12       /* size beyond a stated maximum */
+} omni_status;
+
+typedef enum { OMNI_BSP = 0, OMNI_ASP = 1 } omni_mode;
+typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
+
+/* omni_config.flags */
+#define OMNI_UNSCALED_MEAN 1u   /* lambda_k = 1/K: the unweighted arm of the paper's "weighted aggregation" table */
+#define OMNI_ASP_NO_LR_SCALE 2u /* eta_k = eta: the "w/o LR scaling" arm of the paper's ASP table */
+#define OMNI_INPUT_IS_TIME 4u   /* measurements are compute times t_k instead of throughputs T_k */
+
+/* The "Input:" line of Algorithm 1 / Algorithm 2 (K, B, Delta b_k, b_min, b_max) plus the EWMA weight. */
+typedef struct {
+    int32_t K;            /* workers, 1..OMNI_MAX_K */
+    int32_t global_batch; /* B; initial b_k = B / K (first B mod K workers take one more) */
+    int32_t b_min, b_max; /* batch-size bounds, 1 <= b_min <= b_max */
+    double deadband;      /* Delta b_k of Eq. 7 as a fraction, >= 0 */
+    double ewma_alpha;    /* weight of the newest compute-time sample, (0, 1]; 1 = no smoothing */
+    int32_t mode;         /* OMNI_BSP: Eq. 8 keeps sum b_k = B.  OMNI_ASP: no such rule. */
+    uint32_t flags;
+} omni_config;
+
+/* One bucket = contiguous storage holding one or more whole tensors.  A flat model is one bucket. */
+typedef struct {
+    void *param;              /* device, float[n], 16-byte aligned, read and written: master parameters theta */
+    void *momentum;           /* device, float[n], 16-byte aligned, read and written: v.  May be NULL iff momentum == 0 */
+    void *param_lp;           /* device, bfloat16[n], 16-byte aligned, written: rounded copy of the new theta; or NULL */
+    const void *const *grads; /* HOST array of K device pointers (float[n] or bfloat16[n], 16-byte aligned, read only) */
+    uint64_t n;               /* elements; 0 is allowed (the bucket is skipped) */
+} omni_bucket;
+
+typedef struct {
+    double grad_sqnorm;  /* sum_j gbar_j^2 of the aggregated gradient of the last omni_aggregate_bsp call */
+    double weight_sum;   /* sum_k lambda_k (as rounded to float) of that call */
+    uint64_t steps;      /* synchronous steps enqueued */
+    uint64_t arrivals;   /* asynchronous arrivals enqueued */
+    uint64_t tau_hist[OMNI_TAU_BINS];
+    int32_t tau_max;
+} omni_stats;
+
+typedef struct omni_ctx omni_ctx;
+
+const char *omni_strerror(int status);
+
+/* Create a controller context with b_k = B / K (Algorithm 1, first line of Train).  Needs no GPU.
+ * Errors: NULL, BAD_K, BAD_CONFIG, INFEASIBLE. */
+int omni_create(const omni_config *cfg, omni_ctx **out);
+void omni_destroy(omni_ctx *ctx);
+
+/* Current batch sizes, b[K] host array (BSP: the controller's b_k; ASP: the server's wrkB map). */
+int omni_get_batches(const omni_ctx *ctx, int32_t *b);
+/* Overwrite them.  BAD_BATCH if some b_k < 1 or, in BSP mode, sum != B. */
+int omni_set_batches(omni_ctx *ctx, const int32_t *b);
+
+/* Synchronous re-batch: getAvgComputeTime + getBsz for every worker (Algorithm 1) + Eq. 8.
+ * measured[K] (host): throughput T_k in samples per time unit seen with the current b_k, or the
+ * compute time t_k if OMNI_INPUT_IS_TIME.  Steps, all in IEEE double, sums in ascending k:
+ *   t_k = b_k / T_k;  s_k = EWMA(t_k);  tbar = (sum s_k) / K;                      (Eq. 6a)
+ *   b*_k = b_k - (b_k / s_k) (s_k - tbar);                                          (Eq. 6b)
+ *   if |(b*_k - b_k) / b*_k| >= deadband: b*_k clamped to [b_min, b_max], else b_k;  (Eq. 7)
+ *   round half up to an integer; BSP: shift all workers not pinned at a bound, one unit at a
+ *   time, until sum = B; leftover units go to the largest batches, lowest index first.  (Eq. 8)
+ * new_b[K] (host, out) receives the batches; changed[K] (host, out, may be NULL) 0/1 flags.
+ * Errors: NULL, BAD_MEASUREMENT, INFEASIBLE. */
+int omni_rebatch(omni_ctx *ctx, const double *measured, int32_t *new_b, int32_t *changed);
+
+/* Asynchronous re-batch: evalBsz of Algorithm 2.  Worker `worker` reports the batch it ran and
+ * its measurement; both are stored.  Until every worker has reported once, *new_b_k = b_used.
+ * Afterwards getBsz is re-evaluated for all K stored entries against their mean time (no Eq. 8)
+ * and *new_b_k is the caller's entry.  Errors: NULL, BAD_WORKER, BAD_BATCH, BAD_MEASUREMENT. */
+int omni_asp_report(omni_ctx *ctx, int32_t worker, int32_t b_used, double measured, int32_t *new_b_k);
+
+/* Static variable batching, Eq. 4a: b_k = c_k / sum(c) * B from worker capacities c_k (host,
+ * K positive values, e.g. core counts), rounded to integers within the bounds with sum = B in
+ * BSP mode.  Stores and returns the batches.  Errors: NULL, BAD_MEASUREMENT, INFEASIBLE. */
+int omni_rebatch_static(omni_ctx *ctx, const double *capacity, int32_t *new_b);
+
+/* One synchronous step over all buckets: Eq. 4b/4c fused with the optimiser update.  Per element j:
+ *   lambda_k = float(b_k / sum_i b_i)          (1/K with OMNI_UNSCALED_MEAN)
+ *   gbar = fma(lambda_{K-1}, g_{K-1,j}, ... fma(lambda_0, g_{0,j}, 0))   ascending k, single precision
+ *   d = weight_decay ? fma(weight_decay, theta_j, gbar) : gbar
+ *   v_j = momentum ? fma(momentum, v_j, d) : d          (stored when the momentum buffer is given)
+ *   theta_j = fma(-lr, v_j, theta_j);  param_lp_j = bfloat16(theta_j) round-to-nearest-even
+ * and the squared norm of gbar over all buckets is left in the context (omni_get_stats).
+ * buckets: host array of n_buckets descriptors; b: host int32[K], the batches these gradients
+ * were computed with (each >= 1; in BSP mode sum must equal B).  grad_dtype selects float or
+ * bfloat16 gradients (bfloat16 is widened exactly).  Enqueues on `stream`, does not synchronise.
+ * Errors: NULL, BAD_BATCH, ALIGN, BAD_CONFIG (n_buckets < 0, bad dtype, momentum != 0 with a
+ * NULL momentum buffer), CUDA. */
+int omni_aggregate_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                       const int32_t *b, float lr, float momentum, float weight_decay, void *stream);
+
+/* One asynchronous arrival: worker `worker`'s gradient (buckets[i].grads[worker]), computed on
+ * b_used samples, is applied to the server parameters with eta_k = float(lr * b_used / B)
+ * (Eq. 5b; eta_k = lr with OMNI_ASP_NO_LR_SCALE):
+ *   d = weight_decay ? fma(weight_decay, theta_j, g_j) : g_j;  v_j = momentum ? fma(momentum, v_j, d) : d;
+ *   theta_j = fma(-eta_k, v_j, theta_j)
+ * tau = server updates since this worker last read the parameters; the paper defines no
+ * staleness-dependent factor, so tau is only tallied (omni_stats.tau_hist, tau_max).
+ * Errors: NULL, BAD_WORKER, BAD_BATCH (b_used < 1), BAD_TAU, ALIGN, BAD_CONFIG, CUDA. */
+int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                   int32_t worker, int32_t b_used, int32_t tau, float lr, float momentum, float weight_decay,
+                   void *stream);
+
+/* Same step as omni_aggregate_bsp for gradients that arrive in HOST memory (pinned memory gives
+ * asynchronous copies).  host_grads: host array of n_buckets*K host pointers, entry [i*K + k] =
+ * worker k's gradient for bucket i.  buckets[i].grads must point at K device staging buffers of
+ * n elements each, owned by the caller; the call copies every host gradient into its staging
+ * buffer on `stream`, runs the fused step, copies the squared gradient norm back, synchronises
+ * the stream and stores it in *grad_sqnorm (host, may be NULL).
+ * Errors: as omni_aggregate_bsp. */
+int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                            const void *const *host_grads, const int32_t *b, float lr, float momentum,
+                            float weight_decay, void *stream, double *grad_sqnorm);
+
+/* Synchronises `stream` and fills *out (host). */
+int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream);
+
+/* The cudaError_t of the last failed CUDA call made through this context (0 if none). */
+int omni_last_cuda_error(const omni_ctx *ctx);
+
+/* Persistent-grid size (thread blocks) the synchronous kernel for this K and dtype is launched
+ * with on the current device, and the number of kernels enqueued so far through this context. */
+int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *grid, int32_t *block);
+uint64_t omni_kernel_launches(const omni_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMNI_H_ */

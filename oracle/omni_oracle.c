@@ -207,6 +207,33 @@ int oracle_rebatch(oracle_ctl *c, const double *measured, int32_t *new_b, int32_
     return ORACLE_OK;
 }
 
+/* Static variable batching, Eq. 4a: b_k = c_k / sum_i c_i * K b, with K b the global batch B and
+ * c_k the compute capacity of worker k (cores, FLOPs).
+ * reading: the real-valued shares become integers the same way as in the dynamic controller
+ * (clamp to the bounds, round half up, then the global-batch rule in synchronous mode). */
+int oracle_rebatch_static(oracle_ctl *c, const double *capacity, int32_t *new_b)
+{
+    double csum = 0.0;
+    int32_t n[ORACLE_MAX_K];
+    for (int k = 0; k < c->K; ++k) {
+        if (!isfinite(capacity[k]) || !(capacity[k] > 0.0)) return ORACLE_ERR_MEASUREMENT;
+        csum += capacity[k];
+    }
+    for (int k = 0; k < c->K; ++k) {
+        double x = capacity[k] / csum * (double)c->B;
+        double r = floor(x + 0.5);
+        if (r < (double)c->b_min) r = (double)c->b_min;
+        if (r > (double)c->b_max) r = (double)c->b_max;
+        n[k] = (int32_t)r;
+    }
+    if (c->mode == ORACLE_MODE_BSP) {
+        int rc = conserve_global_batch(c, n);
+        if (rc != ORACLE_OK) return rc;
+    }
+    for (int k = 0; k < c->K; ++k) { c->b[k] = n[k]; new_b[k] = n[k]; }
+    return ORACLE_OK;
+}
+
 /* evalBsz of Alg. 2: worker k reports the batch it ran and its measurement; the server stores
  * both, and once every worker has an entry it re-evaluates getBsz for all K entries against the
  * mean stored time and returns the caller's entry.  No global-batch rule (Sec. IV-D, ASP).

@@ -53,6 +53,7 @@ def lib() -> C.CDLL:
         L.oracle_ctl_get_batches.restype = None
         L.oracle_rebatch.argtypes = [vp, vp, vp, vp, vp]
         L.oracle_asp_report.argtypes = [vp, i32, i32, f64, vp]
+        L.oracle_rebatch_static.argtypes = [vp, vp, vp]
         L.oracle_bsp_weights.argtypes = [i32, vp, u32, vp, vp]
         L.oracle_bsp_weights.restype = None
         L.oracle_asp_lr.argtypes = [f64, i32, i32, u32]
@@ -138,6 +139,15 @@ class Controller:
         if rc != OK:
             raise OracleError(rc)
         return (nb, ch, bs) if want_bstar else (nb, ch)
+
+    def rebatch_static(self, capacity) -> np.ndarray:
+        c = np.ascontiguousarray(capacity, np.float64)
+        assert c.shape == (self.K,)
+        nb = np.zeros(self.K, np.int32)
+        rc = lib().oracle_rebatch_static(self._buf, _ptr(c), _ptr(nb))
+        if rc != OK:
+            raise OracleError(rc)
+        return nb
 
     def asp_report(self, worker, b_used, measured) -> int:
         out = C.c_int32(0)

@@ -1,0 +1,258 @@
+"""Python face of the C-ABI library (``include/omni.h``): argument marshalling only.
+
+Every step of the path runs inside ``libomni.so``; this module turns torch tensors into the
+plain pointers and sizes the C functions take.  There is no fallback: if the library cannot
+be built or loaded, importing a symbol from it raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+from . import build as _build
+
+MAX_K = 32
+TAU_BINS = 33
+BSP, ASP = 0, 1
+F32, BF16 = 0, 1
+UNSCALED_MEAN, ASP_NO_LR_SCALE, INPUT_IS_TIME = 1, 2, 4
+
+OK = 0
+ERR_NULL, ERR_BAD_K, ERR_BAD_WORKER, ERR_BAD_BATCH, ERR_INFEASIBLE, ERR_BAD_MEASUREMENT = -1, -2, -3, -4, -5, -6
+ERR_ALIGN, ERR_BAD_TAU, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_CONFIG, ERR_TOO_LARGE = -7, -8, -9, -10, -11, -12
+
+EXPORTS = (
+    "omni_strerror", "omni_create", "omni_destroy", "omni_get_batches", "omni_set_batches",
+    "omni_rebatch", "omni_asp_report", "omni_rebatch_static", "omni_aggregate_bsp",
+    "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
+    "omni_query_launch", "omni_kernel_launches",
+)
+
+
+class omni_config(C.Structure):
+    _fields_ = [("K", C.c_int32), ("global_batch", C.c_int32), ("b_min", C.c_int32), ("b_max", C.c_int32),
+                ("deadband", C.c_double), ("ewma_alpha", C.c_double), ("mode", C.c_int32), ("flags", C.c_uint32)]
+
+
+class omni_bucket(C.Structure):
+    _fields_ = [("param", C.c_void_p), ("momentum", C.c_void_p), ("param_lp", C.c_void_p),
+                ("grads", C.POINTER(C.c_void_p)), ("n", C.c_uint64)]
+
+
+class omni_stats(C.Structure):
+    _fields_ = [("grad_sqnorm", C.c_double), ("weight_sum", C.c_double), ("steps", C.c_uint64),
+                ("arrivals", C.c_uint64), ("tau_hist", C.c_uint64 * TAU_BINS), ("tau_max", C.c_int32)]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Build (if stale) and load ``libomni.so``; declare the C signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    L = C.CDLL(str(_build.build()))
+    vp, i32, f32 = C.c_void_p, C.c_int32, C.c_float
+    L.omni_strerror.restype = C.c_char_p
+    L.omni_strerror.argtypes = [C.c_int]
+    L.omni_create.argtypes = [C.POINTER(omni_config), C.POINTER(vp)]
+    L.omni_destroy.argtypes = [vp]
+    L.omni_destroy.restype = None
+    L.omni_get_batches.argtypes = [vp, C.POINTER(i32)]
+    L.omni_set_batches.argtypes = [vp, C.POINTER(i32)]
+    L.omni_rebatch.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32), C.POINTER(i32)]
+    L.omni_asp_report.argtypes = [vp, i32, i32, C.c_double, C.POINTER(i32)]
+    L.omni_rebatch_static.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
+    L.omni_aggregate_bsp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(i32), f32, f32, f32, vp]
+    L.omni_apply_asp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, f32, f32, f32, vp]
+    L.omni_aggregate_bsp_host.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(vp), C.POINTER(i32),
+                                          f32, f32, f32, vp, C.POINTER(C.c_double)]
+    L.omni_get_stats.argtypes = [vp, C.POINTER(omni_stats), vp]
+    L.omni_last_cuda_error.argtypes = [vp]
+    L.omni_query_launch.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
+    L.omni_kernel_launches.argtypes = [vp]
+    L.omni_kernel_launches.restype = C.c_uint64
+    _lib = L
+    return L
+
+
+class OmniError(RuntimeError):
+    def __init__(self, status: int, cuda: int = 0):
+        msg = lib().omni_strerror(status).decode()
+        super().__init__(f"omni status {status}: {msg}" + (f" (cudaError {cuda})" if cuda else ""))
+        self.status = status
+        self.cuda = cuda
+
+
+def _dtype_code(t) -> int:
+    import torch
+
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"gradient dtype {t.dtype} is not float32 or bfloat16")
+
+
+@dataclass
+class Stats:
+    grad_sqnorm: float
+    weight_sum: float
+    steps: int
+    arrivals: int
+    tau_hist: List[int]
+    tau_max: int
+
+
+class BucketSet:
+    """Marshalled bucket descriptors, built once and reused every step.
+
+    ``params`` / ``momenta`` / ``params_lp``: one tensor per bucket (momentum and low-precision
+    entries may be None); ``grads[i][k]``: worker k's gradient tensor for bucket i.  The tensors
+    are kept alive by this object.
+    """
+
+    def __init__(self, params: Sequence, grads: Sequence[Sequence], momenta: Optional[Sequence] = None,
+                 params_lp: Optional[Sequence] = None):
+        nb = len(params)
+        momenta = list(momenta) if momenta is not None else [None] * nb
+        params_lp = list(params_lp) if params_lp is not None else [None] * nb
+        assert len(grads) == nb and len(momenta) == nb and len(params_lp) == nb
+        self._keep = (list(params), [list(g) for g in grads], momenta, params_lp)
+        self.n_buckets = nb
+        self.K = len(grads[0]) if nb else 0
+        self.dtype = _dtype_code(grads[0][0]) if nb else F32
+        self.array = (omni_bucket * max(nb, 1))()
+        self._tables = []
+        for i in range(nb):
+            p, m, lp, gs = params[i], momenta[i], params_lp[i], grads[i]
+            n = p.numel()
+            assert p.is_contiguous() and p.dtype.is_floating_point and p.element_size() == 4
+            assert len(gs) == self.K
+            tab = (C.c_void_p * self.K)()
+            for k, g in enumerate(gs):
+                assert g.numel() == n and g.is_contiguous() and _dtype_code(g) == self.dtype
+                tab[k] = g.data_ptr()
+            self._tables.append(tab)
+            if m is not None:
+                assert m.numel() == n and m.is_contiguous() and m.element_size() == 4
+            if lp is not None:
+                assert lp.numel() == n and lp.is_contiguous() and lp.element_size() == 2
+            self.array[i] = omni_bucket(p.data_ptr(), m.data_ptr() if m is not None else None,
+                                        lp.data_ptr() if lp is not None else None,
+                                        C.cast(tab, C.POINTER(C.c_void_p)), n)
+
+    @classmethod
+    def from_flat(cls, layout, theta, grads, v=None, theta_lp=None) -> "BucketSet":
+        """Slice flat buffers (``workloads.Layout``) into per-bucket views."""
+        sl = [slice(b.start, b.start + b.n) for b in layout.buckets]
+        return cls([theta[s] for s in sl], [[g[s] for g in grads] for s in sl],
+                   [v[s] for s in sl] if v is not None else None,
+                   [theta_lp[s] for s in sl] if theta_lp is not None else None)
+
+
+class Omni:
+    """One controller + aggregation context (``omni_ctx``)."""
+
+    def __init__(self, K: int, global_batch: int, b_min: int, b_max: int, deadband: float = 0.10,
+                 ewma_alpha: float = 1.0, mode: int = BSP, flags: int = 0):
+        self._h = C.c_void_p()
+        self.K = K
+        self.global_batch = global_batch
+        cfg = omni_config(K, global_batch, b_min, b_max, deadband, ewma_alpha, mode, flags)
+        self._check(lib().omni_create(C.byref(cfg), C.byref(self._h)))
+        self._i32K = C.c_int32 * K
+        self._f64K = C.c_double * K
+
+    def _check(self, rc: int) -> None:
+        if rc != OK:
+            raise OmniError(rc, lib().omni_last_cuda_error(self._h) if self._h else 0)
+
+    def close(self) -> None:
+        if self._h:
+            lib().omni_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- controller -------------------------------------------------------------------------
+    @property
+    def batches(self) -> List[int]:
+        b = self._i32K()
+        self._check(lib().omni_get_batches(self._h, b))
+        return list(b)
+
+    def set_batches(self, b: Sequence[int]) -> None:
+        self._check(lib().omni_set_batches(self._h, self._i32K(*b)))
+
+    def rebatch(self, measured: Sequence[float]):
+        """Returns (new batches, changed flags)."""
+        nb, ch = self._i32K(), self._i32K()
+        self._check(lib().omni_rebatch(self._h, self._f64K(*measured), nb, ch))
+        return list(nb), list(ch)
+
+    def asp_report(self, worker: int, b_used: int, measured: float) -> int:
+        out = C.c_int32()
+        self._check(lib().omni_asp_report(self._h, worker, b_used, measured, C.byref(out)))
+        return out.value
+
+    def rebatch_static(self, capacity: Sequence[float]) -> List[int]:
+        nb = self._i32K()
+        self._check(lib().omni_rebatch_static(self._h, self._f64K(*capacity), nb))
+        return list(nb)
+
+    # ---- device path ------------------------------------------------------------------------
+    @staticmethod
+    def _stream(stream) -> C.c_void_p:
+        if stream is None:
+            import torch
+
+            stream = torch.cuda.current_stream()
+        return C.c_void_p(stream.cuda_stream)
+
+    def aggregate_bsp(self, buckets: BucketSet, b: Sequence[int], lr: float, momentum: float = 0.0,
+                      weight_decay: float = 0.0, stream=None) -> None:
+        self._check(lib().omni_aggregate_bsp(self._h, buckets.array, buckets.n_buckets, buckets.dtype,
+                                             self._i32K(*b), lr, momentum, weight_decay, self._stream(stream)))
+
+    def aggregate_bsp_host(self, buckets: BucketSet, host_grads: Sequence[Sequence], b: Sequence[int], lr: float,
+                           momentum: float = 0.0, weight_decay: float = 0.0, stream=None) -> float:
+        """``host_grads[i][k]``: pinned host tensor with worker k's gradient of bucket i."""
+        flat = (C.c_void_p * max(1, buckets.n_buckets * self.K))()
+        for i, row in enumerate(host_grads):
+            for k, t in enumerate(row):
+                flat[i * self.K + k] = t.data_ptr()
+        sq = C.c_double()
+        self._check(lib().omni_aggregate_bsp_host(self._h, buckets.array, buckets.n_buckets, buckets.dtype, flat,
+                                                  self._i32K(*b), lr, momentum, weight_decay,
+                                                  self._stream(stream), C.byref(sq)))
+        return sq.value
+
+    def apply_asp(self, buckets: BucketSet, worker: int, b_used: int, tau: int, lr: float, momentum: float = 0.0,
+                  weight_decay: float = 0.0, stream=None) -> None:
+        self._check(lib().omni_apply_asp(self._h, buckets.array, buckets.n_buckets, buckets.dtype, worker, b_used,
+                                         tau, lr, momentum, weight_decay, self._stream(stream)))
+
+    def stats(self, stream=None) -> Stats:
+        s = omni_stats()
+        st = C.c_void_p(0) if stream is None and not self._device_used() else self._stream(stream)
+        self._check(lib().omni_get_stats(self._h, C.byref(s), st))
+        return Stats(s.grad_sqnorm, s.weight_sum, s.steps, s.arrivals, list(s.tau_hist), s.tau_max)
+
+    def _device_used(self) -> bool:
+        return lib().omni_kernel_launches(self._h) > 0
+
+    def query_launch(self, K: int, dtype: int):
+        g, b = C.c_int32(), C.c_int32()
+        self._check(lib().omni_query_launch(self._h, K, dtype, C.byref(g), C.byref(b)))
+        return g.value, b.value
+
+    @property
+    def kernel_launches(self) -> int:
+        return lib().omni_kernel_launches(self._h)

@@ -1,0 +1,428 @@
+// C ABI of the library: context, argument validation, weights, kernel launches.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "controller.h"
+#include "kernels.cuh"
+
+namespace omni {
+
+using KernelFn = const void *;
+
+struct LaunchShape { int grid = 0; int block = kThreads; };
+
+}  // namespace omni
+
+struct omni_ctx {
+    explicit omni_ctx(const omni_config &c) : ctl(c) {}
+    omni::BatchController ctl;
+    omni_stats tally{};
+    omni::Workspace *ws = nullptr;   // device
+    double *host_cell = nullptr;     // pinned, receives the squared norm
+    int device = -1;
+    int sm_count = 0;
+    int last_cuda = 0;
+    uint64_t launches = 0;
+    omni::LaunchShape bsp_shape[2][OMNI_MAX_K + 1];
+    omni::LaunchShape asp_shape[2];
+};
+
+namespace omni {
+namespace {
+
+#define OMNI_CUDA(ctx, call)                         \
+    do {                                             \
+        const cudaError_t e_ = (call);               \
+        if (e_ != cudaSuccess) {                     \
+            (ctx)->last_cuda = int(e_);              \
+            return OMNI_ERR_CUDA;                    \
+        }                                            \
+    } while (0)
+
+template <typename G, int K> KernelFn bsp_fn() { return reinterpret_cast<KernelFn>(&bsp_fused_kernel<G, K>); }
+
+template <typename G> KernelFn bsp_kernel_for(int K)
+{
+    switch (K) {
+#define OMNI_CASE(k) case k: return bsp_fn<G, k>();
+        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
+        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
+        OMNI_CASE(17) OMNI_CASE(18) OMNI_CASE(19) OMNI_CASE(20) OMNI_CASE(21) OMNI_CASE(22) OMNI_CASE(23) OMNI_CASE(24)
+        OMNI_CASE(25) OMNI_CASE(26) OMNI_CASE(27) OMNI_CASE(28) OMNI_CASE(29) OMNI_CASE(30) OMNI_CASE(31) OMNI_CASE(32)
+#undef OMNI_CASE
+    }
+    return nullptr;
+}
+
+KernelFn bsp_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bsp_kernel_for<__nv_bfloat16>(K) : bsp_kernel_for<float>(K); }
+KernelFn asp_kernel(int dtype)
+{
+    return dtype == OMNI_BF16 ? reinterpret_cast<KernelFn>(&asp_apply_kernel<__nv_bfloat16>)
+                              : reinterpret_cast<KernelFn>(&asp_apply_kernel<float>);
+}
+
+unsigned long long bsp_tile_elems(int dtype, int K)
+{
+    return (unsigned long long)kThreads * (dtype == OMNI_BF16 ? 8 : 4) * bsp_unroll(K);
+}
+unsigned long long asp_tile_elems(int dtype) { return (unsigned long long)kThreads * (dtype == OMNI_BF16 ? 8 : 4) * kAspUnroll; }
+
+// First kernel-launching call of a context: bind to the current device, allocate the workspace.
+int ensure_device(omni_ctx *ctx)
+{
+    if (ctx->ws) {
+        int cur = -1;
+        OMNI_CUDA(ctx, cudaGetDevice(&cur));
+        if (cur != ctx->device) return OMNI_ERR_BAD_CONFIG;
+        return OMNI_OK;
+    }
+    int dev = -1;
+    OMNI_CUDA(ctx, cudaGetDevice(&dev));
+    OMNI_CUDA(ctx, cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    Workspace *ws = nullptr;
+    OMNI_CUDA(ctx, cudaMalloc(&ws, sizeof(Workspace)));
+    cudaError_t e = cudaMemset(ws, 0, sizeof(Workspace));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->host_cell, sizeof(double));
+    if (e != cudaSuccess) {
+        cudaFree(ws);
+        ctx->last_cuda = int(e);
+        return OMNI_ERR_CUDA;
+    }
+    *ctx->host_cell = 0.0;
+    ctx->ws = ws;
+    ctx->device = dev;
+    return OMNI_OK;
+}
+
+// Persistent grid = SM count x resident CTAs per SM of that kernel, capped by the slot count.
+int shape_for(omni_ctx *ctx, KernelFn fn, LaunchShape &s)
+{
+    if (s.grid > 0) return OMNI_OK;
+    int per_sm = 0;
+    OMNI_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, 0));
+    if (per_sm < 1) per_sm = 1;
+    int grid = ctx->sm_count * per_sm;
+    if (grid > kMaxGrid) grid = kMaxGrid / ctx->sm_count * ctx->sm_count;
+    s.grid = grid;
+    return OMNI_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks shared by the synchronous and asynchronous entry points.  worker < 0: all K gradients.
+int check_buckets(const omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t dtype, int worker,
+                  float momentum)
+{
+    if (n_buckets < 0 || (dtype != OMNI_F32 && dtype != OMNI_BF16)) return OMNI_ERR_BAD_CONFIG;
+    if (n_buckets > 0 && !buckets) return OMNI_ERR_NULL;
+    if (!std::isfinite(momentum)) return OMNI_ERR_BAD_CONFIG;
+    const int K = ctx->ctl.K();
+    for (int i = 0; i < n_buckets; ++i) {
+        const omni_bucket &b = buckets[i];
+        if (b.n == 0) continue;
+        if (!b.param || !b.grads) return OMNI_ERR_NULL;
+        if (momentum != 0.0f && !b.momentum) return OMNI_ERR_BAD_CONFIG;
+        if (!aligned16(b.param) || !aligned16(b.momentum) || !aligned16(b.param_lp)) return OMNI_ERR_ALIGN;
+        for (int k = (worker < 0 ? 0 : worker); k < (worker < 0 ? K : worker + 1); ++k) {
+            if (!b.grads[k]) return OMNI_ERR_NULL;
+            if (!aligned16(b.grads[k])) return OMNI_ERR_ALIGN;
+        }
+    }
+    return OMNI_OK;
+}
+
+int launch(omni_ctx *ctx, KernelFn fn, int grid, void *params, cudaStream_t stream)
+{
+    void *args[] = {params};
+    OMNI_CUDA(ctx, cudaLaunchKernel(fn, dim3(grid), dim3(kThreads), args, 0, stream));
+    ctx->launches += 1;
+    return OMNI_OK;
+}
+
+// Eq. 4b: lambda_k = b_k / sum b, evaluated in double and rounded once to float.
+double fill_weights(const omni_ctx *ctx, const int32_t *b, float *lam)
+{
+    const int K = ctx->ctl.K();
+    int64_t total = 0;
+    for (int k = 0; k < K; ++k) total += b[k];
+    double wsum = 0.0;
+    for (int k = 0; k < K; ++k) {
+        const double l = (ctx->ctl.config().flags & OMNI_UNSCALED_MEAN) ? 1.0 / double(K) : double(b[k]) / double(total);
+        lam[k] = float(l);
+        wsum += double(lam[k]);
+    }
+    return wsum;
+}
+
+int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t dtype, const float *lam,
+                float lr, float mu, float wd, cudaStream_t stream)
+{
+    const int K = ctx->ctl.K();
+    KernelFn fn = bsp_kernel(dtype, K);
+    LaunchShape &shape = ctx->bsp_shape[dtype][K];
+    int rc = shape_for(ctx, fn, shape);
+    if (rc != OMNI_OK) return rc;
+    const unsigned long long tile = bsp_tile_elems(dtype, K);
+
+    BspParams p;
+    int launched = 0, i = 0;
+    while (i < n_buckets || launched == 0) {
+        std::memset(&p, 0, sizeof p);
+        unsigned long long tiles = 0;
+        int nb = 0;
+        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+            const omni_bucket &b = buckets[i];
+            if (b.n == 0) continue;
+            p.bk[nb] = {static_cast<float *>(b.param), static_cast<float *>(b.momentum),
+                        static_cast<__nv_bfloat16 *>(b.param_lp), b.n, tiles};
+            for (int k = 0; k < K; ++k) p.g[nb][k] = b.grads[k];
+            tiles += (b.n + tile - 1) / tile;
+            ++nb;
+        }
+        // an empty call still runs one (empty) launch so that the squared norm reads 0
+        for (int k = 0; k < K; ++k) p.lam[k] = lam[k];
+        p.lr = lr; p.mu = mu; p.wd = wd;
+        p.nb = nb;
+        p.accumulate = launched > 0;
+        p.tiles = tiles;
+        p.ws = ctx->ws;
+        const unsigned long long want = tiles < 1 ? 1 : tiles;
+        const int grid = want < (unsigned long long)shape.grid ? int(want) : shape.grid;
+        rc = launch(ctx, fn, grid, &p, stream);
+        if (rc != OMNI_OK) return rc;
+        ++launched;
+    }
+    return OMNI_OK;
+}
+
+}  // namespace
+}  // namespace omni
+
+using namespace omni;
+
+extern "C" {
+
+const char *omni_strerror(int s)
+{
+    switch (s) {
+        case OMNI_OK: return "ok";
+        case OMNI_ERR_NULL: return "a required pointer is NULL";
+        case OMNI_ERR_BAD_K: return "K outside 1..32";
+        case OMNI_ERR_BAD_WORKER: return "worker index out of range";
+        case OMNI_ERR_BAD_BATCH: return "batch size < 1 or batch sizes do not sum to the global batch";
+        case OMNI_ERR_INFEASIBLE: return "bounds cannot hold the global batch";
+        case OMNI_ERR_BAD_MEASUREMENT: return "measurement not finite or not positive";
+        case OMNI_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case OMNI_ERR_BAD_TAU: return "negative staleness";
+        case OMNI_ERR_CUDA: return "CUDA call failed (see omni_last_cuda_error)";
+        case OMNI_ERR_TIMEOUT: return "device-side wait ran out";
+        case OMNI_ERR_BAD_CONFIG: return "invalid configuration or argument";
+        case OMNI_ERR_TOO_LARGE: return "size beyond the stated maximum";
+    }
+    return "unknown status";
+}
+
+int omni_create(const omni_config *cfg, omni_ctx **out)
+{
+    if (!cfg || !out) return OMNI_ERR_NULL;
+    const int rc = BatchController::validate(*cfg);
+    if (rc != OMNI_OK) return rc;
+    omni_ctx *ctx = new (std::nothrow) omni_ctx(*cfg);
+    if (!ctx) return OMNI_ERR_CUDA;
+    ctx->tally.tau_max = 0;
+    *out = ctx;
+    return OMNI_OK;
+}
+
+void omni_destroy(omni_ctx *ctx)
+{
+    if (!ctx) return;
+    if (ctx->ws) cudaFree(ctx->ws);
+    if (ctx->host_cell) cudaFreeHost(ctx->host_cell);
+    delete ctx;
+}
+
+int omni_get_batches(const omni_ctx *ctx, int32_t *b)
+{
+    if (!ctx || !b) return OMNI_ERR_NULL;
+    std::memcpy(b, ctx->ctl.batches(), sizeof(int32_t) * ctx->ctl.K());
+    return OMNI_OK;
+}
+
+int omni_set_batches(omni_ctx *ctx, const int32_t *b)
+{
+    if (!ctx || !b) return OMNI_ERR_NULL;
+    return ctx->ctl.set_batches(b);
+}
+
+int omni_rebatch(omni_ctx *ctx, const double *measured, int32_t *new_b, int32_t *changed)
+{
+    if (!ctx || !measured || !new_b) return OMNI_ERR_NULL;
+    return ctx->ctl.rebatch(measured, new_b, changed);
+}
+
+int omni_asp_report(omni_ctx *ctx, int32_t worker, int32_t b_used, double measured, int32_t *new_b_k)
+{
+    if (!ctx || !new_b_k) return OMNI_ERR_NULL;
+    return ctx->ctl.report(worker, b_used, measured, new_b_k);
+}
+
+int omni_rebatch_static(omni_ctx *ctx, const double *capacity, int32_t *new_b)
+{
+    if (!ctx || !capacity || !new_b) return OMNI_ERR_NULL;
+    return ctx->ctl.rebatch_static(capacity, new_b);
+}
+
+static int check_bsp_batches(const omni_ctx *ctx, const int32_t *b)
+{
+    int64_t total = 0;
+    for (int k = 0; k < ctx->ctl.K(); ++k) {
+        if (b[k] < 1) return OMNI_ERR_BAD_BATCH;
+        total += b[k];
+    }
+    if (ctx->ctl.config().mode == OMNI_BSP && total != ctx->ctl.B()) return OMNI_ERR_BAD_BATCH;
+    return OMNI_OK;
+}
+
+int omni_aggregate_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                       const int32_t *b, float lr, float momentum, float weight_decay, void *stream)
+{
+    if (!ctx || !b) return OMNI_ERR_NULL;
+    int rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, -1, momentum);
+    if (rc != OMNI_OK) return rc;
+    rc = check_bsp_batches(ctx, b);
+    if (rc != OMNI_OK) return rc;
+    rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    float lam[OMNI_MAX_K];
+    const double wsum = fill_weights(ctx, b, lam);
+    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, lr, momentum, weight_decay,
+                     static_cast<cudaStream_t>(stream));
+    if (rc != OMNI_OK) return rc;
+    ctx->tally.weight_sum = wsum;
+    ctx->tally.steps += 1;
+    return OMNI_OK;
+}
+
+int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                            const void *const *host_grads, const int32_t *b, float lr, float momentum,
+                            float weight_decay, void *stream, double *grad_sqnorm)
+{
+    if (!ctx || !b || (n_buckets > 0 && !host_grads)) return OMNI_ERR_NULL;
+    int rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, -1, momentum);
+    if (rc != OMNI_OK) return rc;
+    rc = check_bsp_batches(ctx, b);
+    if (rc != OMNI_OK) return rc;
+    const int K = ctx->ctl.K();
+    for (int i = 0; i < n_buckets; ++i)
+        for (int k = 0; k < K && buckets[i].n; ++k)
+            if (!host_grads[size_t(i) * K + k]) return OMNI_ERR_NULL;
+    rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esz = grad_dtype == OMNI_BF16 ? 2 : 4;
+    for (int i = 0; i < n_buckets; ++i)
+        for (int k = 0; k < K && buckets[i].n; ++k)
+            OMNI_CUDA(ctx, cudaMemcpyAsync(const_cast<void *>(buckets[i].grads[k]), host_grads[size_t(i) * K + k],
+                                           buckets[i].n * esz, cudaMemcpyHostToDevice, s));
+    float lam[OMNI_MAX_K];
+    const double wsum = fill_weights(ctx, b, lam);
+    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, lr, momentum, weight_decay, s);
+    if (rc != OMNI_OK) return rc;
+    ctx->tally.weight_sum = wsum;
+    ctx->tally.steps += 1;
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->host_cell, &ctx->ws->sqnorm, sizeof(double), cudaMemcpyDeviceToHost, s));
+    OMNI_CUDA(ctx, cudaStreamSynchronize(s));
+    if (grad_sqnorm) *grad_sqnorm = *ctx->host_cell;
+    return OMNI_OK;
+}
+
+int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                   int32_t worker, int32_t b_used, int32_t tau, float lr, float momentum, float weight_decay,
+                   void *stream)
+{
+    if (!ctx) return OMNI_ERR_NULL;
+    const int K = ctx->ctl.K();
+    if (worker < 0 || worker >= K) return OMNI_ERR_BAD_WORKER;
+    if (b_used < 1) return OMNI_ERR_BAD_BATCH;
+    if (tau < 0) return OMNI_ERR_BAD_TAU;
+    int rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, worker, momentum);
+    if (rc != OMNI_OK) return rc;
+    rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+
+    // Eq. 5b: eta_k = eta * b_k / B, in double, rounded once to float
+    const double eta_k = (ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
+                             ? double(lr)
+                             : double(lr) * double(b_used) / double(ctx->ctl.B());
+    KernelFn fn = asp_kernel(grad_dtype);
+    LaunchShape &shape = ctx->asp_shape[grad_dtype];
+    rc = shape_for(ctx, fn, shape);
+    if (rc != OMNI_OK) return rc;
+    const unsigned long long tile = asp_tile_elems(grad_dtype);
+
+    AspParams p;
+    int i = 0;
+    while (i < n_buckets) {
+        std::memset(&p, 0, sizeof p);
+        unsigned long long tiles = 0;
+        int nb = 0;
+        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+            const omni_bucket &bk = buckets[i];
+            if (bk.n == 0) continue;
+            p.bk[nb] = {static_cast<float *>(bk.param), static_cast<float *>(bk.momentum),
+                        static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
+            p.g[nb] = bk.grads[worker];
+            tiles += (bk.n + tile - 1) / tile;
+            ++nb;
+        }
+        if (nb == 0) break;
+        p.eta = float(eta_k); p.mu = momentum; p.wd = weight_decay;
+        p.nb = nb;
+        p.tiles = tiles;
+        const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
+        rc = launch(ctx, fn, grid, &p, static_cast<cudaStream_t>(stream));
+        if (rc != OMNI_OK) return rc;
+    }
+    ctx->tally.arrivals += 1;
+    ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
+    if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+    return OMNI_OK;
+}
+
+int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream)
+{
+    if (!ctx || !out) return OMNI_ERR_NULL;
+    if (ctx->ws) {
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->host_cell, &ctx->ws->sqnorm, sizeof(double), cudaMemcpyDeviceToHost, s));
+        OMNI_CUDA(ctx, cudaStreamSynchronize(s));
+        ctx->tally.grad_sqnorm = *ctx->host_cell;
+    }
+    *out = ctx->tally;
+    return OMNI_OK;
+}
+
+int omni_last_cuda_error(const omni_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *grid, int32_t *block)
+{
+    if (!ctx || !grid || !block) return OMNI_ERR_NULL;
+    if (K < 1 || K > OMNI_MAX_K) return OMNI_ERR_BAD_K;
+    if (grad_dtype != OMNI_F32 && grad_dtype != OMNI_BF16) return OMNI_ERR_BAD_CONFIG;
+    int rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    LaunchShape &shape = ctx->bsp_shape[grad_dtype][K];
+    rc = shape_for(ctx, bsp_kernel(grad_dtype, K), shape);
+    if (rc != OMNI_OK) return rc;
+    *grid = shape.grid;
+    *block = shape.block;
+    return OMNI_OK;
+}
+
+uint64_t omni_kernel_launches(const omni_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,430 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle, element by
+element on the same seeded inputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2503_17469_b200 import binding as B
+from paper_2503_17469_b200 import workloads as W
+
+from parity_util import Guarded, SQNORM_RTOL, assert_close, to_np
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _gen(seed):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    return g
+
+
+def _make(K, n, kind, seed, lp=False, momentum=True, gstd=1e-3):
+    gen = _gen(seed)
+    gdt = torch.bfloat16 if kind == "bf16" else torch.float32
+    theta = Guarded(n, torch.float32, DEV, torch.empty(n, device=DEV).normal_(0, 0.05, generator=gen))
+    v = Guarded(n, torch.float32, DEV, torch.zeros(n, device=DEV)) if momentum else None
+    grads = [Guarded(n, gdt, DEV, torch.empty(n, device=DEV).normal_(0, gstd, generator=gen).to(gdt)) for _ in range(K)]
+    plp = Guarded(n, torch.bfloat16, DEV, torch.zeros(n, device=DEV, dtype=torch.bfloat16)) if lp else None
+    return theta, v, grads, plp
+
+
+def _random_batches(K, per, seed):
+    rng = np.random.default_rng(seed)
+    if K == 1:
+        return [per]
+    cuts = np.sort(rng.choice(np.arange(1, K * per), K - 1, replace=False))
+    b = np.diff(np.concatenate([[0], cuts, [K * per]]))
+    return [int(x) for x in b]
+
+
+SIZES = [1, 3, 7, 1023, 4095, 4097, 3 * 8192 + 17, 100_003]
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 5, 8, 11, 16, 17, 32])
+def test_bsp_flat_parity_over_sizes(K, kind):
+    """Several tiles plus a ragged tail, three steps each, momentum + weight decay + low-precision copy."""
+    bit_equal = []
+    for n in SIZES:
+        theta, v, grads, plp = _make(K, n, kind, 1000 * K + n % 997, lp=True)
+        b = _random_batches(K, 32, K + n)
+        o = B.Omni(K, 32 * K, 1, 32 * K, 0.1)
+        bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t], [plp.t])
+        th_o, v_o = to_np(theta.t), to_np(v.t)
+        lp_o = np.zeros(n, np.uint16)
+        g_np = [to_np(g.t) for g in grads]
+        for step in range(3):
+            o.aggregate_bsp(bs, b, 0.1, 0.9, 5e-4)
+            sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 5e-4, theta_lp=lp_o)
+            st = o.stats()
+            assert abs(st.grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o + 1e-300
+            assert st.steps == step + 1
+        bit_equal.append(assert_close(to_np(theta.t), th_o, kind, f"theta K={K} n={n}"))
+        bit_equal.append(assert_close(to_np(v.t), v_o, kind, f"v K={K} n={n}"))
+        assert np.array_equal(to_np(plp.t), lp_o)
+        for buf in (theta, v, plp, *grads):
+            assert buf.intact(), "guard band overwritten"
+        for g, g0 in zip(grads, g_np):
+            assert np.array_equal(to_np(g.t), g0), "gradient buffer modified"
+    # both sides are the same ordered chain of correctly rounded FMAs
+    assert min(bit_equal) == 1.0
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+@pytest.mark.parametrize("mu,wd,with_v", [(0.0, 0.0, False), (0.0, 0.0, True), (0.9, 0.0, True), (0.0, 1e-3, False)])
+def test_bsp_update_variants(kind, mu, wd, with_v):
+    K, n = 4, 50_001
+    theta, v, grads, _ = _make(K, n, kind, 77, momentum=with_v)
+    b = [3, 9, 20, 32]
+    o = B.Omni(K, 64, 1, 64, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t] if with_v else None)
+    th_o = to_np(theta.t)
+    v_o = to_np(v.t) if with_v else None
+    g_np = [to_np(g.t) for g in grads]
+    for _ in range(2):
+        o.aggregate_bsp(bs, b, 0.05, mu, wd)
+        O.bsp_step_f32(g_np, b, th_o, v_o, 0.05, mu, wd)
+    assert assert_close(to_np(theta.t), th_o, kind) == 1.0
+    if with_v:
+        assert assert_close(to_np(v.t), v_o, kind) == 1.0
+
+
+def test_bsp_against_double_definition():
+    """Ten steps against the double-precision oracle at the contract tolerance."""
+    K, n = 16, 200_003
+    theta, v, grads, _ = _make(K, n, "f32", 5)
+    b = _random_batches(K, 32, 5)
+    o = B.Omni(K, 512, 1, 512, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    th64, v64 = to_np(theta.t).astype(np.float64), np.zeros(n)
+    g_np = [to_np(g.t) for g in grads]
+    for _ in range(10):
+        o.aggregate_bsp(bs, b, 0.1, 0.9, 0.0)
+        sq64 = O.bsp_step_f64(g_np, b, th64, v64, 0.1, 0.9, 0.0)
+    np.testing.assert_allclose(to_np(theta.t), th64, rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(to_np(v.t), v64, rtol=1e-5, atol=1e-8)
+    assert abs(o.stats().grad_sqnorm - sq64) <= SQNORM_RTOL * sq64
+
+
+def test_unscaled_mean_flag_and_equal_batches():
+    K, n = 8, 30_000
+    theta, v, grads, _ = _make(K, n, "f32", 9)
+    g_np = [to_np(g.t) for g in grads]
+    th0 = to_np(theta.t)
+    o = B.Omni(K, 256, 1, 256, 0.1, flags=B.UNSCALED_MEAN)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    b = _random_batches(K, 32, 9)
+    o.aggregate_bsp(bs, b, 1.0, 0.0, 0.0)
+    th_o = th0.copy()
+    O.bsp_step_f32(g_np, b, th_o, None, 1.0, 0.0, 0.0, flags=O.FLAG_UNSCALED_MEAN)
+    assert np.array_equal(to_np(theta.t), th_o)
+    # equal batches without the flag give the same bits (lambda = 1/8 exactly)
+    theta.t.copy_(torch.from_numpy(th0))
+    o2 = B.Omni(K, 256, 1, 256, 0.1)
+    o2.aggregate_bsp(bs, [32] * K, 1.0, 0.0, 0.0)
+    assert np.array_equal(to_np(theta.t), th_o)
+    assert o2.stats().weight_sum == 1.0
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+def test_bsp_many_buckets_empty_and_ragged(kind):
+    """23 buckets (three launches of at most 8), some empty, odd sizes, per-bucket momentum/lp mix."""
+    K = 5
+    rng = np.random.default_rng(3)
+    sizes = [int(x) for x in rng.choice([0, 1, 5, 300, 2048, 6144, 10_007, 40_001], 23)]
+    sizes[0], sizes[7], sizes[22] = 0, 0, 12_345
+    o = B.Omni(K, 160, 1, 160, 0.1)
+    b = _random_batches(K, 32, 1)
+    bufs, params, moms, lps, gl = [], [], [], [], []
+    for i, n in enumerate(sizes):
+        theta, v, grads, plp = _make(K, max(n, 1), kind, 500 + i, lp=(i % 2 == 0))
+        bufs.append((theta, v, grads, plp, n))
+        params.append(theta.t[:n]); moms.append(v.t[:n]); gl.append([g.t[:n] for g in grads])
+        lps.append(plp.t[:n] if plp is not None else None)
+    bs = B.BucketSet(params, gl, moms, lps)
+    oracle_state = [(to_np(p), to_np(m), [to_np(g) for g in gs]) for p, m, gs in zip(params, moms, gl)]
+    before = o.kernel_launches
+    o.aggregate_bsp(bs, b, 0.1, 0.9, 1e-4)
+    assert o.kernel_launches - before == 3
+    sq_total = 0.0
+    for (theta, v, grads, plp, n), (th_o, v_o, g_np) in zip(bufs, oracle_state):
+        lp_o = np.zeros(n, np.uint16)
+        if n:
+            sq_total += O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 1e-4, theta_lp=lp_o)
+        assert np.array_equal(to_np(theta.t[:n]), th_o) and np.array_equal(to_np(v.t[:n]), v_o)
+        if plp is not None:
+            assert np.array_equal(to_np(plp.t[:n]), lp_o)
+        assert theta.intact() and v.intact() and (plp is None or plp.intact())
+        if n == 0:   # an empty bucket leaves its storage alone
+            assert float(v.t[0]) == 0.0
+    assert abs(o.stats().grad_sqnorm - sq_total) <= SQNORM_RTOL * sq_total
+
+
+def test_empty_call_reads_zero_norm():
+    o = B.Omni(2, 64, 4, 96, 0.1)
+    theta, v, grads, _ = _make(2, 1000, "f32", 1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    o.aggregate_bsp(bs, [32, 32], 0.1, 0.9)
+    assert o.stats().grad_sqnorm > 0
+    empty = B.BucketSet([], [])
+    empty.K, empty.dtype = 2, B.F32
+    o.aggregate_bsp(empty, [32, 32], 0.1, 0.9)
+    assert o.stats().grad_sqnorm == 0.0
+
+
+def test_results_are_deterministic():
+    K, n = 16, 1_000_003
+    outs = []
+    for rep in range(2):
+        theta, v, grads, _ = _make(K, n, "bf16", 42)
+        o = B.Omni(K, 512, 1, 512, 0.1)
+        bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+        for _ in range(3):
+            o.aggregate_bsp(bs, _random_batches(K, 32, 4), 0.1, 0.9)
+        outs.append((to_np(theta.t), o.stats().grad_sqnorm))
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+
+
+def test_host_gradient_entry_point():
+    K, n = 4, 70_001
+    theta, v, grads, _ = _make(K, n, "bf16", 11)
+    host = [[g.t.cpu().pin_memory() for g in grads]]
+    g_np = [to_np(g.t) for g in grads]
+    for g in grads:
+        g.t.zero_()                      # staging buffers: the call must fill them
+    th_o, v_o = to_np(theta.t), to_np(v.t)
+    o = B.Omni(K, 128, 4, 96, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    b = [10, 20, 30, 68]
+    sq = o.aggregate_bsp_host(bs, host, b, 0.1, 0.9)
+    sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 0.0)
+    assert abs(sq - sq_o) <= SQNORM_RTOL * sq_o
+    assert np.array_equal(to_np(theta.t), th_o) and np.array_equal(to_np(v.t), v_o)
+
+
+# ------------------------------------------------------------------------------------------------
+# asynchronous arrivals
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+@pytest.mark.parametrize("mu,wd", [(0.0, 0.0), (0.9, 1e-4)])
+def test_asp_parity_over_sizes(kind, mu, wd):
+    K = 3
+    for n in SIZES + [4 * 8192 * 3 + 5]:
+        theta, v, grads, plp = _make(K, n, kind, 2000 + n % 991, lp=True, momentum=mu != 0)
+        o = B.Omni(K, 96, 4, 96, 0.1, 1.0, B.ASP)
+        bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t] if v else None, [plp.t])
+        th_o = to_np(theta.t)
+        v_o = to_np(v.t) if v else None
+        lp_o = np.zeros(n, np.uint16)
+        g_np = [to_np(g.t) for g in grads]
+        taus = []
+        for i, (k, b_used, tau) in enumerate([(0, 32, 0), (2, 7, 3), (1, 96, 40), (2, 33, 1)]):
+            o.apply_asp(bs, k, b_used, tau, 0.1, mu, wd)
+            O.asp_apply_f32(g_np[k], b_used, 96, th_o, v_o, 0.1, mu, wd, theta_lp=lp_o)
+            taus.append(tau)
+        assert assert_close(to_np(theta.t), th_o, kind, f"n={n}") == 1.0
+        if v:
+            assert assert_close(to_np(v.t), v_o, kind) == 1.0
+        assert np.array_equal(to_np(plp.t), lp_o)
+        assert theta.intact() and plp.intact() and all(g.intact() for g in grads)
+        st = o.stats()
+        ref = O.TauStats()
+        for t in taus:
+            ref.record(t)
+        assert st.arrivals == 4 and st.tau_hist == ref.hist.tolist() and st.tau_max == ref.tau_max
+
+
+def test_asp_no_lr_scale_flag():
+    n = 10_000
+    theta, _, grads, _ = _make(2, n, "f32", 8, momentum=False)
+    o = B.Omni(2, 64, 4, 96, 0.1, 1.0, B.ASP, B.ASP_NO_LR_SCALE)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]])
+    th_o = to_np(theta.t)
+    o.apply_asp(bs, 1, 8, 0, 0.1)
+    O.asp_apply_f32(to_np(grads[1].t), 8, 64, th_o, None, 0.1, 0.0, 0.0, flags=O.FLAG_ASP_NO_LR_SCALE)
+    assert np.array_equal(to_np(theta.t), th_o)
+
+
+def _asp_stream(cfg, n_events, apply_fn, report_fn, seed):
+    """Throughput-weighted arrival stream with controller feedback (the workload recipe):
+    worker drawn with probability proportional to its iteration rate T_k / b_k; staleness =
+    server updates since that worker's previous arrival."""
+    gen = torch.Generator().manual_seed(seed)
+    T = W.draw_throughputs(cfg.K, gen, cfg.ratio)
+    u = torch.rand(n_events, generator=gen, dtype=torch.float64).tolist()
+    b = [cfg.global_batch // cfg.K] * cfg.K
+    last = [0] * cfg.K
+    trace = []
+    for i in range(n_events):
+        k = W.pick_worker(u[i], [T[j] / b[j] for j in range(cfg.K)])
+        tau = min(i - last[k], 10**6)
+        apply_fn(k, b[k], tau)
+        last[k] = i + 1
+        b[k] = report_fn(k, b[k], T[k])
+        trace.append((k, tau, b[k]))
+    return trace
+
+
+def test_asp_event_stream_with_controller_feedback():
+    """The asynchronous configuration on a shrunk model: 1000 arrivals, every arrival applied
+    and reported on both sides; batches and staleness tallies bit-exact, parameters at tolerance."""
+    cfg = W.scaled(W.config("resnet50_asp"), 600)
+    buf = W.make_buffers(cfg, DEV)
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.ASP)
+    bs = B.BucketSet.from_flat(buf.layout, buf.theta, buf.grads)
+    ora = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, O.MODE_ASP)
+    th_o = to_np(buf.theta)
+    g_np = [to_np(g) for g in buf.grads]
+    tally = O.TauStats()
+
+    def ora_apply(k, b_used, tau):
+        O.asp_apply_f32(g_np[k], b_used, cfg.global_batch, th_o, None, cfg.lr, 0.0, 0.0)
+        tally.record(tau)
+
+    t_lib = _asp_stream(cfg, 1000, lambda k, bu, tau: o.apply_asp(bs, k, bu, tau, cfg.lr), o.asp_report, cfg.seed)
+    t_ora = _asp_stream(cfg, 1000, ora_apply, ora.asp_report, cfg.seed)
+    assert t_lib == t_ora
+    st = o.stats()
+    assert st.arrivals == 1000 and st.tau_hist == tally.hist.tolist() and st.tau_max == tally.tau_max
+    assert o.batches == ora.batches.tolist()
+    assert assert_close(to_np(buf.theta), th_o, "f32") == 1.0
+
+
+# ------------------------------------------------------------------------------------------------
+# the synthetic configurations
+# ------------------------------------------------------------------------------------------------
+
+def test_tiny_config_every_step():
+    """K=4, 2^20 parameters: one re-batch (expected (2,6,19,37)) then 10 steps, parity at every step."""
+    cfg = W.config("tiny")
+    buf = W.make_buffers(cfg, DEV)
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
+    ora = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
+    b, _ = o.rebatch(cfg.throughputs)
+    assert b == ora.rebatch(cfg.throughputs)[0].tolist() == [2, 6, 19, 37]
+    bs = B.BucketSet.from_flat(buf.layout, buf.theta, buf.grads, buf.v)
+    th_o, v_o, g_np = to_np(buf.theta), to_np(buf.v), [to_np(g) for g in buf.grads]
+    for step in range(cfg.steps):
+        o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum)
+        sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, cfg.lr, cfg.momentum, 0.0)
+        assert assert_close(to_np(buf.theta), th_o, "f32", f"step {step}") == 1.0
+        assert assert_close(to_np(buf.v), v_o, "f32", f"step {step}") == 1.0
+        assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+
+
+def _bsp_config_run(name, steps, numel_cap=None, lp=False):
+    cfg = W.config(name)
+    if numel_cap:
+        cfg = W.scaled(cfg, numel_cap)
+    buf = W.make_buffers(cfg, DEV)
+    lay = buf.layout
+    theta_lp = torch.zeros(lay.total, dtype=torch.bfloat16, device=DEV) if lp else None
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
+    ora = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
+    bs = B.BucketSet.from_flat(lay, buf.theta, buf.grads, buf.v, theta_lp)
+    gen = torch.Generator().manual_seed(cfg.seed)
+    base = W.draw_throughputs(cfg.K, gen, cfg.ratio)
+    th_o, v_o, g_np = to_np(buf.theta), to_np(buf.v), [to_np(g) for g in buf.grads]
+    lp_o = np.zeros(lay.total, np.uint16) if lp else None
+    b = o.batches
+    for step in range(steps):
+        if step % max(cfg.rebatch_every, 1) == 0 and (cfg.rebatch_every or step == 0):
+            T = W.jitter_throughputs(W.interference(base, step) if name == "vgg16" else base, gen)
+            b, _ = o.rebatch(T)
+            assert b == ora.rebatch(T)[0].tolist() and sum(b) == cfg.global_batch
+        o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+        # the oracle walks the same buckets (padding elements are zeros on both sides)
+        sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, cfg.lr, cfg.momentum, cfg.weight_decay, theta_lp=lp_o)
+        assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+    kind = cfg.grad_dtype
+    assert assert_close(to_np(buf.theta), th_o, kind, name) == 1.0
+    assert assert_close(to_np(buf.v), v_o, kind, name) == 1.0
+    if lp:
+        assert np.array_equal(to_np(theta_lp), lp_o)
+    return o
+
+
+def test_resnet18_config_shrunk_full_schedule():
+    """62 tensors, 2 buckets, K=8, 100 steps with a re-batch every 10 (tensors capped at 3000 elements)."""
+    _bsp_config_run("resnet18", 100, numel_cap=3000)
+
+
+def test_resnet18_config_full_size():
+    _bsp_config_run("resnet18", 12)
+
+
+def test_resnet50_bf16_config_full_size():
+    """The headline configuration at full size, 3 steps with the low-precision copy."""
+    o = _bsp_config_run("resnet50_bf16", 3, lp=True)
+    grid, block = o.query_launch(16, B.BF16)
+    assert grid % torch.cuda.get_device_properties(0).multi_processor_count == 0 and block == 256
+
+
+def test_resnet50_f32_config_full_size():
+    _bsp_config_run("resnet50_f32", 2)
+
+
+def test_vgg16_config_shrunk_with_interference_phase():
+    """K=32, 32 tensors, re-batch every step through the interference phase (steps 15-34)."""
+    _bsp_config_run("vgg16", 50, numel_cap=5000)
+
+
+def _sample_blocks(total, rng, n_blocks=48, width=4096):
+    starts = sorted(int(s) for s in rng.integers(0, max(total - width, 1), n_blocks))
+    return [(s, min(s + width, total)) for s in starts]
+
+
+def test_vgg16_config_full_size_sampled():
+    """K=32, 138M parameters, 7 buckets: two steps at full size; the oracle recomputes sampled
+    blocks (the rules are element-wise, so a block needs only its own inputs) including every
+    bucket's first and last elements; the squared norm is checked against its expectation for
+    i.i.d. gradients, sigma^2 * sum(lambda^2) * P."""
+    cfg = W.config("vgg16")
+    buf = W.make_buffers(cfg, DEV)
+    lay = buf.layout
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
+    gen = torch.Generator().manual_seed(cfg.seed)
+    T = W.draw_throughputs(cfg.K, gen, cfg.ratio)
+    b, _ = o.rebatch(T)
+    bs = B.BucketSet.from_flat(lay, buf.theta, buf.grads, buf.v)
+    rng = np.random.default_rng(cfg.seed)
+    blocks = _sample_blocks(lay.total, rng)
+    for bk in lay.buckets:
+        blocks += [(bk.start, min(bk.start + 300, bk.start + bk.n)), (max(bk.start, bk.start + bk.n - 300), bk.start + bk.n)]
+    snap = [(to_np(buf.theta[s:e]), to_np(buf.v[s:e]), [to_np(g[s:e]) for g in buf.grads]) for s, e in blocks]
+    for _ in range(2):
+        o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum)
+    for (s, e), (th_o, v_o, g_np) in zip(blocks, snap):
+        for _ in range(2):
+            O.bsp_step_f32(g_np, b, th_o, v_o, cfg.lr, cfg.momentum, 0.0)
+        assert np.array_equal(to_np(buf.theta[s:e]), th_o), (s, e)
+        assert np.array_equal(to_np(buf.v[s:e]), v_o), (s, e)
+    lam = O.bsp_weights(b)[0]
+    expect = cfg.grad_std ** 2 * float((lam ** 2).sum()) * cfg.P
+    assert abs(o.stats().grad_sqnorm - expect) <= 0.01 * expect
+
+
+def test_resnet50_asp_full_size_sampled():
+    """25.6M parameters, 20 arrivals at full size against the oracle on sampled blocks."""
+    cfg = W.config("resnet50_asp")
+    buf = W.make_buffers(cfg, DEV)
+    lay = buf.layout
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, 1.0, B.ASP)
+    bs = B.BucketSet.from_flat(lay, buf.theta, buf.grads)
+    rng = np.random.default_rng(cfg.seed)
+    blocks = _sample_blocks(lay.total, rng)
+    for bk in lay.buckets:
+        blocks += [(bk.start, bk.start + 300), (bk.start + bk.n - 300, bk.start + bk.n)]
+    snap = [(to_np(buf.theta[s:e]), [to_np(g[s:e]) for g in buf.grads]) for s, e in blocks]
+    events = []
+    _asp_stream(cfg, 20, lambda k, bu, tau: (events.append((k, bu, tau)), o.apply_asp(bs, k, bu, tau, cfg.lr)),
+                o.asp_report, cfg.seed)
+    for (s, e), (th_o, g_np) in zip(blocks, snap):
+        for k, bu, tau in events:
+            O.asp_apply_f32(g_np[k], bu, cfg.global_batch, th_o, None, cfg.lr, 0.0, 0.0)
+        assert np.array_equal(to_np(buf.theta[s:e]), th_o), (s, e)

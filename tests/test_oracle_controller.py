@@ -226,3 +226,19 @@ def test_errors_leave_state_untouched():
 def test_initial_batches_when_k_does_not_divide_b():
     c = O.Controller(3, 64, 1, 64, 0.1)
     assert c.batches.tolist() == [22, 21, 21]
+
+
+def test_static_variable_batching_by_capacity():
+    """Eq. 4a with the core counts of Table I: shares of B proportional to cores."""
+    c = O.Controller(4, 128, 4, 96, 0.1)
+    assert c.rebatch_static([12, 12, 12, 12]).tolist() == [32, 32, 32, 32]      # HL1
+    assert c.rebatch_static([6, 6, 4, 32]).tolist() == [16, 16, 11, 85]         # BSP HL8: 16, 16, 10.67, 85.33
+    assert c.rebatch_static([10, 10, 6, 22]).tolist() == [27, 27, 16, 58]       # 26.67->27, 16, 58.67->59: 1 over, from the largest
+    c3 = O.Controller(3, 64, 1, 64, 0.1)
+    assert c3.rebatch_static([1, 1, 1]).tolist() == [22, 21, 21]                # 21.33 each, one unit short -> lowest index
+    rng = np.random.default_rng(7)
+    for _ in range(100):
+        K = int(rng.integers(2, 17))
+        cc = O.Controller(K, 32 * K, 4, 96, 0.1)
+        nb = cc.rebatch_static(rng.uniform(1, 8, K))
+        assert nb.sum() == 32 * K and nb.min() >= 4 and nb.max() <= 96
