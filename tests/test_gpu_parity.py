@@ -132,7 +132,7 @@ def test_unscaled_mean_flag_and_equal_batches():
 
 @pytest.mark.parametrize("kind", ["f32", "bf16"])
 def test_bsp_many_buckets_empty_and_ragged(kind):
-    """23 buckets (three launches of at most 8), some empty, odd sizes, per-bucket momentum/lp mix."""
+    """23 buckets (several launches of at most 8 non-empty ones), some empty, odd sizes, mixed lp."""
     K = 5
     rng = np.random.default_rng(3)
     sizes = [int(x) for x in rng.choice([0, 1, 5, 300, 2048, 6144, 10_007, 40_001], 23)]
@@ -149,7 +149,7 @@ def test_bsp_many_buckets_empty_and_ragged(kind):
     oracle_state = [(to_np(p), to_np(m), [to_np(g) for g in gs]) for p, m, gs in zip(params, moms, gl)]
     before = o.kernel_launches
     o.aggregate_bsp(bs, b, 0.1, 0.9, 1e-4)
-    assert o.kernel_launches - before == 3
+    assert o.kernel_launches - before == math.ceil(sum(1 for n in sizes if n) / 8) >= 2
     sq_total = 0.0
     for (theta, v, grads, plp, n), (th_o, v_o, g_np) in zip(bufs, oracle_state):
         lp_o = np.zeros(n, np.uint16)
