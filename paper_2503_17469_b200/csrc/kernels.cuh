@@ -3,10 +3,16 @@
 // The work is HBM-bound: per parameter a synchronous step reads K gradient values plus theta and
 // v and writes theta and v (4K+16 bytes in float, 2K+16 with bfloat16 gradients); an
 // asynchronous arrival moves 12 or 20 bytes.  There is no data reuse and no contraction, so the
-// design goal is bytes in flight: every thread issues all of its 128-bit loads (K gradient
-// streams, theta, v) before the first dependent FMA, the grid is persistent (a multiple of the
-// SM count) and walks tiles with a grid stride so that neighbouring CTAs touch neighbouring
-// DRAM pages, and loads/stores carry streaming cache hints because nothing is read twice.
+// design goal is bytes in flight and DRAM-friendly request shapes:
+//   - every thread issues all of its loads (K gradient streams, theta, v) before the first
+//     dependent FMA;
+//   - loads and stores are 256 bits wide (ld/st.global.v8.b32, new with sm_100) whenever all
+//     buffers are 32-byte aligned, so one warp instruction covers 1 KB of one stream; a 128-bit
+//     variant serves buffers that are only 16-byte aligned;
+//   - nothing is read twice, so gradient loads go through the non-coherent path without L1
+//     allocation and everything is marked evict-first in L2;
+//   - the grid is persistent (SM count x resident CTAs) and walks tiles with a grid stride, so
+//     that at any moment the whole GPU sweeps one narrow window of each stream.
 //
 // Arithmetic is the ordered single-precision FMA chain documented in omni.h; the worker loop is
 // unrolled at compile time (K is a template argument) so the chain order is fixed in the code.
@@ -20,7 +26,6 @@
 
 namespace omni {
 
-constexpr int kThreads = 256;            // threads per CTA
 constexpr int kMaxBucketsPerLaunch = 8;  // bucket descriptors carried in the kernel parameters
 constexpr int kMaxGrid = 148 * 16;       // upper bound of the persistent grid = partial-sum slots
 
@@ -59,57 +64,123 @@ struct AspParams {
     unsigned long long tiles;
 };
 
-// Elements one thread handles per 128-bit gradient load.
-template <typename G> struct Vec { static constexpr int n = 16 / sizeof(G); };
-
-// How many 128-bit vectors per stream a thread keeps in flight: small K gets more so that the
-// bytes in flight per SM stay high.
-__host__ __device__ constexpr int bsp_unroll(int K) { return K <= 2 ? 4 : K <= 5 ? 3 : K <= 10 ? 2 : 1; }
-constexpr int kAspUnroll = 4;
-
-template <typename G> __host__ __device__ constexpr unsigned long long bsp_tile(int K)
+// ---------------------------------------------------------------------------------------------
+// Launch shape per (gradient type, K): threads per CTA and gradient vectors per thread and
+// stream.  Chosen from timing sweeps on B200; the rule keeps roughly 0.4-0.6 KB of loads per
+// thread in flight.
+// ---------------------------------------------------------------------------------------------
+template <typename G> __host__ __device__ constexpr int bsp_threads(int K)
 {
-    return (unsigned long long)kThreads * Vec<G>::n * bsp_unroll(K);
+    return sizeof(G) == 2 && K >= 12 ? 192 : 256;
 }
-template <typename G> __host__ __device__ constexpr unsigned long long asp_tile()
-{
-    return (unsigned long long)kThreads * Vec<G>::n * kAspUnroll;
-}
+template <typename G> __host__ __device__ constexpr int bsp_chunks(int K) { return K <= 2 ? 4 : K <= 10 ? 2 : 1; }
+constexpr int kAspThreads = 256;
+constexpr int kAspChunks = 2;
 
 // ---------------------------------------------------------------------------------------------
-// loads / stores with streaming hints
+// 128- and 256-bit global memory access with streaming hints
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 ld_stream(const void *p) { return __ldcs(reinterpret_cast<const uint4 *>(p)); }
-__device__ __forceinline__ void st_stream(void *p, uint4 x) { __stcs(reinterpret_cast<uint4 *>(p), x); }
-__device__ __forceinline__ void st_stream(void *p, uint2 x) { __stcs(reinterpret_cast<uint2 *>(p), x); }
+template <int WORDS> struct Raw { unsigned w[WORDS]; };
 
-__device__ __forceinline__ float bf16_lo(unsigned w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(unsigned w) { return __uint_as_float(w & 0xffff0000u); }
+// read-only stream (gradients): non-coherent path
+template <int WORDS> __device__ __forceinline__ Raw<WORDS> ld_ro(const void *p)
+{
+    Raw<WORDS> r;
+    if constexpr (WORDS == 8)
+        asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]), "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+                     : "l"(p));
+    else {
+        const uint4 x = __ldcs(reinterpret_cast<const uint4 *>(p));
+        r.w[0] = x.x; r.w[1] = x.y; r.w[2] = x.z; r.w[3] = x.w;
+    }
+    return r;
+}
+// buffers this kernel also writes (theta, v): coherent path
+template <int WORDS> __device__ __forceinline__ Raw<WORDS> ld_rw(const void *p)
+{
+    Raw<WORDS> r;
+    if constexpr (WORDS == 8)
+        asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r.w[0]), "=r"(r.w[1]), "=r"(r.w[2]), "=r"(r.w[3]), "=r"(r.w[4]), "=r"(r.w[5]), "=r"(r.w[6]), "=r"(r.w[7])
+                     : "l"(p) : "memory");
+    else {
+        const uint4 x = __ldcs(reinterpret_cast<const uint4 *>(p));
+        r.w[0] = x.x; r.w[1] = x.y; r.w[2] = x.z; r.w[3] = x.w;
+    }
+    return r;
+}
+template <int WORDS> __device__ __forceinline__ void st_words(void *p, const unsigned *w)
+{
+    if constexpr (WORDS == 8)
+        asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};"
+                     :: "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]), "l"(p) : "memory");
+    else if constexpr (WORDS == 4)
+        __stcs(reinterpret_cast<uint4 *>(p), make_uint4(w[0], w[1], w[2], w[3]));
+    else
+        __stcs(reinterpret_cast<uint2 *>(p), make_uint2(w[0], w[1]));
+}
 
-// One 128-bit gradient vector -> Vec<G>::n floats.
-template <typename G> __device__ __forceinline__ void widen(const uint4 &r, float *out);
-template <> __device__ __forceinline__ void widen<float>(const uint4 &r, float *o)
+// Vector geometry: one gradient vector is VB bytes = E elements; theta/v need E floats.
+template <typename G, bool WIDE> struct Geo {
+    static constexpr int VB = WIDE ? 32 : 16;
+    static constexpr int GW = VB / 4;               // 32-bit words per gradient vector
+    static constexpr int E = VB / int(sizeof(G));   // elements per vector
+    static constexpr int FW = GW;                   // words per theta/v access (same width)
+    static constexpr int FN = E / FW;               // theta/v accesses per vector (1 for float, 2 for bfloat16)
+    static constexpr int LW = E / 2;                // words of the bfloat16 copy per vector
+};
+
+template <typename G, int GW> __device__ __forceinline__ void widen(const Raw<GW> &r, float *o)
 {
-    o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y);
-    o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
+    if constexpr (sizeof(G) == 4) {
+#pragma unroll
+        for (int i = 0; i < GW; ++i) o[i] = __uint_as_float(r.w[i]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < GW; ++i) {
+            o[2 * i] = __uint_as_float(r.w[i] << 16);
+            o[2 * i + 1] = __uint_as_float(r.w[i] & 0xffff0000u);
+        }
+    }
 }
-template <> __device__ __forceinline__ void widen<__nv_bfloat16>(const uint4 &r, float *o)
+template <typename G> __device__ __forceinline__ float widen1(const G *p, unsigned long long j)
 {
-    o[0] = bf16_lo(r.x); o[1] = bf16_hi(r.x); o[2] = bf16_lo(r.y); o[3] = bf16_hi(r.y);
-    o[4] = bf16_lo(r.z); o[5] = bf16_hi(r.z); o[6] = bf16_lo(r.w); o[7] = bf16_hi(r.w);
-}
-template <typename G> __device__ __forceinline__ float widen1(const G *p, unsigned long long j);
-template <> __device__ __forceinline__ float widen1<float>(const float *p, unsigned long long j) { return __ldcs(p + j); }
-template <> __device__ __forceinline__ float widen1<__nv_bfloat16>(const __nv_bfloat16 *p, unsigned long long j)
-{
-    return __uint_as_float((unsigned)__ldcs(reinterpret_cast<const unsigned short *>(p) + j) << 16);
+    if constexpr (sizeof(G) == 4) return __ldcs(reinterpret_cast<const float *>(p) + j);
+    else return __uint_as_float((unsigned)__ldcs(reinterpret_cast<const unsigned short *>(p) + j) << 16);
 }
 
+template <int FW, int FN> __device__ __forceinline__ void load_floats(const float *p, float *o)
+{
+#pragma unroll
+    for (int i = 0; i < FN; ++i) {
+        const Raw<FW> r = ld_rw<FW>(p + FW * i);
+#pragma unroll
+        for (int j = 0; j < FW; ++j) o[FW * i + j] = __uint_as_float(r.w[j]);
+    }
+}
+template <int FW, int FN> __device__ __forceinline__ void store_floats(float *p, const float *o)
+{
+#pragma unroll
+    for (int i = 0; i < FN; ++i) {
+        unsigned w[FW];
+#pragma unroll
+        for (int j = 0; j < FW; ++j) w[j] = __float_as_uint(o[FW * i + j]);
+        st_words<FW>(p + FW * i, w);
+    }
+}
 __device__ __forceinline__ unsigned pack_bf16(float a, float b)
 {
     const unsigned lo = __bfloat16_as_ushort(__float2bfloat16_rn(a));
     const unsigned hi = __bfloat16_as_ushort(__float2bfloat16_rn(b));
     return lo | (hi << 16);
+}
+template <int LW> __device__ __forceinline__ void store_lp(__nv_bfloat16 *p, const float *o)
+{
+    unsigned w[LW];
+#pragma unroll
+    for (int i = 0; i < LW; ++i) w[i] = pack_bf16(o[2 * i], o[2 * i + 1]);
+    st_words<LW>(p, w);
 }
 
 // The update of one element after gbar is known.  Returns the new theta, writes the new v.
@@ -121,30 +192,6 @@ __device__ __forceinline__ float update_one(float gbar, float theta, float &v, f
     return __fmaf_rn(-lr, vn, theta);
 }
 
-template <int N> __device__ __forceinline__ void load_f32(const float *p, float *o)
-{
-#pragma unroll
-    for (int i = 0; i < N / 4; ++i) {
-        const uint4 r = ld_stream(p + 4 * i);
-        o[4 * i] = __uint_as_float(r.x); o[4 * i + 1] = __uint_as_float(r.y);
-        o[4 * i + 2] = __uint_as_float(r.z); o[4 * i + 3] = __uint_as_float(r.w);
-    }
-}
-template <int N> __device__ __forceinline__ void store_f32(float *p, const float *o)
-{
-#pragma unroll
-    for (int i = 0; i < N / 4; ++i)
-        st_stream(p + 4 * i, make_uint4(__float_as_uint(o[4 * i]), __float_as_uint(o[4 * i + 1]),
-                                        __float_as_uint(o[4 * i + 2]), __float_as_uint(o[4 * i + 3])));
-}
-template <int N> __device__ __forceinline__ void store_lp(__nv_bfloat16 *p, const float *o)
-{
-    if constexpr (N == 8)
-        st_stream(p, make_uint4(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3]), pack_bf16(o[4], o[5]), pack_bf16(o[6], o[7])));
-    else
-        st_stream(p, make_uint2(pack_bf16(o[0], o[1]), pack_bf16(o[2], o[3])));
-}
-
 template <int NB> __device__ __forceinline__ int find_bucket(const BucketDesc *bk, int nb, unsigned long long tile)
 {
     int bi = 0;
@@ -154,15 +201,50 @@ template <int NB> __device__ __forceinline__ int find_bucket(const BucketDesc *b
     return bi;
 }
 
+// Squared-norm epilogue: warp tree, CTA sum in warp order, one partial per CTA; the CTA that
+// takes the last ticket adds the partials in index order, so the result depends only on the
+// grid size.  The ticket is left at zero for the next launch.
+template <int THREADS> __device__ __forceinline__ void finish_sqnorm(double sq, Workspace *ws, int accumulate)
+{
+    __shared__ double wsum[THREADS / 32];
+    __shared__ bool is_last;
+    const int tid = threadIdx.x;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
+    if ((tid & 31) == 0) wsum[tid >> 5] = sq;
+    __syncthreads();
+    if (tid == 0) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < THREADS / 32; ++w) s += wsum[w];
+        ws->partials[blockIdx.x] = s;
+        __threadfence();
+        const unsigned t = atomicAdd(&ws->ticket, 1u);
+        is_last = t == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (is_last && tid < 32) {
+        __threadfence();
+        double s = 0.0;
+        for (unsigned i = tid; i < gridDim.x; i += 32) s += __ldcg(&ws->partials[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+        if (tid == 0) {
+            ws->sqnorm = accumulate ? ws->sqnorm + s : s;
+            ws->ticket = 0u;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Synchronous step: K-way weighted sum + update + squared norm of the aggregate
 // ---------------------------------------------------------------------------------------------
-template <typename G, int K>
-__global__ void __launch_bounds__(kThreads) bsp_fused_kernel(const __grid_constant__ BspParams p)
+template <typename G, int K, int THREADS, int C, bool WIDE>
+__global__ void __launch_bounds__(THREADS) bsp_fused_kernel(const __grid_constant__ BspParams p)
 {
-    constexpr int V = Vec<G>::n;
-    constexpr int U = bsp_unroll(K);
-    constexpr unsigned long long TILE = bsp_tile<G>(K);
+    using Ge = Geo<G, WIDE>;
+    constexpr int E = Ge::E;
+    constexpr unsigned long long TILE = (unsigned long long)THREADS * E * C;
     const int tid = threadIdx.x;
     const float lr = p.lr, mu = p.mu, wd = p.wd;
     double sq = 0.0;
@@ -175,44 +257,44 @@ __global__ void __launch_bounds__(kThreads) bsp_fused_kernel(const __grid_consta
 
         if (base + TILE <= bd.n) {
             // full tile: every load of this thread is issued before the first FMA
-            uint4 raw[U][K];
-            float th[U][V], vv[U][V];
+            Raw<Ge::GW> raw[C][K];
+            float th[C][E], vv[C][E];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const unsigned long long off = base + (unsigned long long)(u * kThreads + tid) * V;
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
 #pragma unroll
-                for (int k = 0; k < K; ++k) raw[u][k] = ld_stream(static_cast<const G *>(p.g[bi][k]) + off);
-                load_f32<V>(bd.theta + off, th[u]);
-                if (mu != 0.0f) load_f32<V>(bd.v + off, vv[u]);
+                for (int k = 0; k < K; ++k) raw[c][k] = ld_ro<Ge::GW>(static_cast<const G *>(p.g[bi][k]) + off);
+                load_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (mu != 0.0f) load_floats<Ge::FW, Ge::FN>(bd.v + off, vv[c]);
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const unsigned long long off = base + (unsigned long long)(u * kThreads + tid) * V;
-                float acc[V];
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                float acc[E];
 #pragma unroll
-                for (int e = 0; e < V; ++e) acc[e] = 0.0f;
+                for (int e = 0; e < E; ++e) acc[e] = 0.0f;
 #pragma unroll
                 for (int k = 0; k < K; ++k) {
-                    float gk[V];
-                    widen<G>(raw[u][k], gk);
+                    float gk[E];
+                    widen<G, Ge::GW>(raw[c][k], gk);
                     const float lam = p.lam[k];
 #pragma unroll
-                    for (int e = 0; e < V; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
+                    for (int e = 0; e < E; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
                 }
                 float part = 0.0f;
 #pragma unroll
-                for (int e = 0; e < V; ++e) {
+                for (int e = 0; e < E; ++e) {
                     part = __fmaf_rn(acc[e], acc[e], part);
-                    th[u][e] = update_one(acc[e], th[u][e], vv[u][e], lr, mu, wd);
+                    th[c][e] = update_one(acc[e], th[c][e], vv[c][e], lr, mu, wd);
                 }
                 sq += (double)part;
-                store_f32<V>(bd.theta + off, th[u]);
-                if (has_v) store_f32<V>(bd.v + off, vv[u]);
-                if (has_lp) store_lp<V>(bd.lp + off, th[u]);
+                store_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (has_v) store_floats<Ge::FW, Ge::FN>(bd.v + off, vv[c]);
+                if (has_lp) store_lp<Ge::LW>(bd.lp + off, th[c]);
             }
         } else {
             // ragged last tile of a bucket: element by element, same arithmetic
-            for (unsigned long long j = base + tid; j < bd.n; j += kThreads) {
+            for (unsigned long long j = base + tid; j < bd.n; j += THREADS) {
                 float acc = 0.0f;
 #pragma unroll
                 for (int k = 0; k < K; ++k)
@@ -226,47 +308,18 @@ __global__ void __launch_bounds__(kThreads) bsp_fused_kernel(const __grid_consta
             }
         }
     }
-
-    // squared norm: warp tree, CTA sum in warp order, one partial per CTA; the CTA that takes the
-    // last ticket adds the partials in index order, so the result depends only on the grid size.
-    __shared__ double wsum[kThreads / 32];
-    __shared__ bool is_last;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sq += __shfl_down_sync(0xffffffffu, sq, o);
-    if ((tid & 31) == 0) wsum[tid >> 5] = sq;
-    __syncthreads();
-    if (tid == 0) {
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) s += wsum[w];
-        p.ws->partials[blockIdx.x] = s;
-        __threadfence();
-        const unsigned t = atomicAdd(&p.ws->ticket, 1u);
-        is_last = t == gridDim.x - 1;
-    }
-    __syncthreads();
-    if (is_last && tid < 32) {
-        __threadfence();
-        double s = 0.0;
-        for (unsigned i = tid; i < gridDim.x; i += 32) s += __ldcg(&p.ws->partials[i]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
-        if (tid == 0) {
-            p.ws->sqnorm = p.accumulate ? p.ws->sqnorm + s : s;
-            p.ws->ticket = 0u;
-        }
-    }
+    finish_sqnorm<THREADS>(sq, p.ws, p.accumulate);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Asynchronous arrival: one gradient stream applied with eta_k
 // ---------------------------------------------------------------------------------------------
-template <typename G>
-__global__ void __launch_bounds__(kThreads) asp_apply_kernel(const __grid_constant__ AspParams p)
+template <typename G, int THREADS, int C, bool WIDE>
+__global__ void __launch_bounds__(THREADS) asp_apply_kernel(const __grid_constant__ AspParams p)
 {
-    constexpr int V = Vec<G>::n;
-    constexpr int U = kAspUnroll;
-    constexpr unsigned long long TILE = asp_tile<G>();
+    using Ge = Geo<G, WIDE>;
+    constexpr int E = Ge::E;
+    constexpr unsigned long long TILE = (unsigned long long)THREADS * E * C;
     const int tid = threadIdx.x;
     const float eta = p.eta, mu = p.mu, wd = p.wd;
 
@@ -278,28 +331,28 @@ __global__ void __launch_bounds__(kThreads) asp_apply_kernel(const __grid_consta
         const bool has_v = bd.v != nullptr, has_lp = bd.lp != nullptr;
 
         if (base + TILE <= bd.n) {
-            uint4 raw[U];
-            float th[U][V], vv[U][V];
+            Raw<Ge::GW> raw[C];
+            float th[C][E], vv[C][E];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const unsigned long long off = base + (unsigned long long)(u * kThreads + tid) * V;
-                raw[u] = ld_stream(g + off);
-                load_f32<V>(bd.theta + off, th[u]);
-                if (mu != 0.0f) load_f32<V>(bd.v + off, vv[u]);
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                raw[c] = ld_ro<Ge::GW>(g + off);
+                load_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (mu != 0.0f) load_floats<Ge::FW, Ge::FN>(bd.v + off, vv[c]);
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const unsigned long long off = base + (unsigned long long)(u * kThreads + tid) * V;
-                float gk[V];
-                widen<G>(raw[u], gk);
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                float gk[E];
+                widen<G, Ge::GW>(raw[c], gk);
 #pragma unroll
-                for (int e = 0; e < V; ++e) th[u][e] = update_one(gk[e], th[u][e], vv[u][e], eta, mu, wd);
-                store_f32<V>(bd.theta + off, th[u]);
-                if (has_v) store_f32<V>(bd.v + off, vv[u]);
-                if (has_lp) store_lp<V>(bd.lp + off, th[u]);
+                for (int e = 0; e < E; ++e) th[c][e] = update_one(gk[e], th[c][e], vv[c][e], eta, mu, wd);
+                store_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (has_v) store_floats<Ge::FW, Ge::FN>(bd.v + off, vv[c]);
+                if (has_lp) store_lp<Ge::LW>(bd.lp + off, th[c]);
             }
         } else {
-            for (unsigned long long j = base + tid; j < bd.n; j += kThreads) {
+            for (unsigned long long j = base + tid; j < bd.n; j += THREADS) {
                 float vj = mu != 0.0f ? __ldcs(bd.v + j) : 0.0f;
                 const float t = update_one(widen1<G>(g, j), __ldcs(bd.theta + j), vj, eta, mu, wd);
                 bd.theta[j] = t;

@@ -12,7 +12,14 @@ namespace omni {
 
 using KernelFn = const void *;
 
-struct LaunchShape { int grid = 0; int block = kThreads; };
+// A kernel instantiation with the launch geometry that goes with it.
+struct KernelInfo {
+    KernelFn fn = nullptr;
+    int threads = 0;
+    unsigned long long tile = 0;  // elements per tile
+};
+
+struct LaunchShape { int grid = 0; int block = 0; };
 
 }  // namespace omni
 
@@ -26,8 +33,8 @@ struct omni_ctx {
     int sm_count = 0;
     int last_cuda = 0;
     uint64_t launches = 0;
-    omni::LaunchShape bsp_shape[2][OMNI_MAX_K + 1];
-    omni::LaunchShape asp_shape[2];
+    omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
+    omni::LaunchShape asp_shape[2][2];                  // [dtype][wide]
 };
 
 namespace omni {
@@ -42,33 +49,42 @@ namespace {
         }                                            \
     } while (0)
 
-template <typename G, int K> KernelFn bsp_fn() { return reinterpret_cast<KernelFn>(&bsp_fused_kernel<G, K>); }
+template <typename G, int K, bool WIDE> KernelInfo bsp_info()
+{
+    constexpr int T = bsp_threads<G>(K), C = bsp_chunks<G>(K);
+    return {reinterpret_cast<KernelFn>(&bsp_fused_kernel<G, K, T, C, WIDE>), T,
+            (unsigned long long)T * Geo<G, WIDE>::E * C};
+}
 
-template <typename G> KernelFn bsp_kernel_for(int K)
+template <typename G, bool WIDE> KernelInfo bsp_kernel_for(int K)
 {
     switch (K) {
-#define OMNI_CASE(k) case k: return bsp_fn<G, k>();
+#define OMNI_CASE(k) case k: return bsp_info<G, k, WIDE>();
         OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
         OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
         OMNI_CASE(17) OMNI_CASE(18) OMNI_CASE(19) OMNI_CASE(20) OMNI_CASE(21) OMNI_CASE(22) OMNI_CASE(23) OMNI_CASE(24)
         OMNI_CASE(25) OMNI_CASE(26) OMNI_CASE(27) OMNI_CASE(28) OMNI_CASE(29) OMNI_CASE(30) OMNI_CASE(31) OMNI_CASE(32)
 #undef OMNI_CASE
     }
-    return nullptr;
+    return {};
 }
 
-KernelFn bsp_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bsp_kernel_for<__nv_bfloat16>(K) : bsp_kernel_for<float>(K); }
-KernelFn asp_kernel(int dtype)
+KernelInfo bsp_kernel(int dtype, int K, bool wide)
 {
-    return dtype == OMNI_BF16 ? reinterpret_cast<KernelFn>(&asp_apply_kernel<__nv_bfloat16>)
-                              : reinterpret_cast<KernelFn>(&asp_apply_kernel<float>);
+    if (dtype == OMNI_BF16) return wide ? bsp_kernel_for<__nv_bfloat16, true>(K) : bsp_kernel_for<__nv_bfloat16, false>(K);
+    return wide ? bsp_kernel_for<float, true>(K) : bsp_kernel_for<float, false>(K);
 }
 
-unsigned long long bsp_tile_elems(int dtype, int K)
+template <typename G, bool WIDE> KernelInfo asp_info()
 {
-    return (unsigned long long)kThreads * (dtype == OMNI_BF16 ? 8 : 4) * bsp_unroll(K);
+    return {reinterpret_cast<KernelFn>(&asp_apply_kernel<G, kAspThreads, kAspChunks, WIDE>), kAspThreads,
+            (unsigned long long)kAspThreads * Geo<G, WIDE>::E * kAspChunks};
 }
-unsigned long long asp_tile_elems(int dtype) { return (unsigned long long)kThreads * (dtype == OMNI_BF16 ? 8 : 4) * kAspUnroll; }
+KernelInfo asp_kernel(int dtype, bool wide)
+{
+    if (dtype == OMNI_BF16) return wide ? asp_info<__nv_bfloat16, true>() : asp_info<__nv_bfloat16, false>();
+    return wide ? asp_info<float, true>() : asp_info<float, false>();
+}
 
 // First kernel-launching call of a context: bind to the current device, allocate the workspace.
 int ensure_device(omni_ctx *ctx)
@@ -98,19 +114,34 @@ int ensure_device(omni_ctx *ctx)
 }
 
 // Persistent grid = SM count x resident CTAs per SM of that kernel, capped by the slot count.
-int shape_for(omni_ctx *ctx, KernelFn fn, LaunchShape &s)
+int shape_for(omni_ctx *ctx, const KernelInfo &ki, LaunchShape &s)
 {
     if (s.grid > 0) return OMNI_OK;
     int per_sm = 0;
-    OMNI_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, 0));
+    OMNI_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ki.fn, ki.threads, 0));
     if (per_sm < 1) per_sm = 1;
     int grid = ctx->sm_count * per_sm;
     if (grid > kMaxGrid) grid = kMaxGrid / ctx->sm_count * ctx->sm_count;
     s.grid = grid;
+    s.block = ki.threads;
     return OMNI_OK;
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+
+// The 256-bit kernels need every buffer of every non-empty bucket on a 32-byte boundary.
+bool all_aligned32(const omni_bucket *buckets, int32_t n_buckets, int k0, int k1)
+{
+    for (int i = 0; i < n_buckets; ++i) {
+        const omni_bucket &b = buckets[i];
+        if (b.n == 0) continue;
+        if (!aligned32(b.param) || !aligned32(b.momentum) || !aligned32(b.param_lp)) return false;
+        for (int k = k0; k < k1; ++k)
+            if (!aligned32(b.grads[k])) return false;
+    }
+    return true;
+}
 
 // Checks shared by the synchronous and asynchronous entry points.  worker < 0: all K gradients.
 int check_buckets(const omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t dtype, int worker,
@@ -134,10 +165,10 @@ int check_buckets(const omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buc
     return OMNI_OK;
 }
 
-int launch(omni_ctx *ctx, KernelFn fn, int grid, void *params, cudaStream_t stream)
+int launch(omni_ctx *ctx, const KernelInfo &ki, int grid, void *params, cudaStream_t stream)
 {
     void *args[] = {params};
-    OMNI_CUDA(ctx, cudaLaunchKernel(fn, dim3(grid), dim3(kThreads), args, 0, stream));
+    OMNI_CUDA(ctx, cudaLaunchKernel(ki.fn, dim3(grid), dim3(ki.threads), args, 0, stream));
     ctx->launches += 1;
     return OMNI_OK;
 }
@@ -161,11 +192,12 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
                 float lr, float mu, float wd, cudaStream_t stream)
 {
     const int K = ctx->ctl.K();
-    KernelFn fn = bsp_kernel(dtype, K);
-    LaunchShape &shape = ctx->bsp_shape[dtype][K];
-    int rc = shape_for(ctx, fn, shape);
+    const bool wide = all_aligned32(buckets, n_buckets, 0, K);
+    const KernelInfo ki = bsp_kernel(dtype, K, wide);
+    LaunchShape &shape = ctx->bsp_shape[dtype][wide][K];
+    int rc = shape_for(ctx, ki, shape);
     if (rc != OMNI_OK) return rc;
-    const unsigned long long tile = bsp_tile_elems(dtype, K);
+    const unsigned long long tile = ki.tile;
 
     BspParams p;
     int launched = 0, i = 0;
@@ -191,7 +223,7 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
         p.ws = ctx->ws;
         const unsigned long long want = tiles < 1 ? 1 : tiles;
         const int grid = want < (unsigned long long)shape.grid ? int(want) : shape.grid;
-        rc = launch(ctx, fn, grid, &p, stream);
+        rc = launch(ctx, ki, grid, &p, stream);
         if (rc != OMNI_OK) return rc;
         ++launched;
     }
@@ -358,11 +390,12 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
     const double eta_k = (ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
                              ? double(lr)
                              : double(lr) * double(b_used) / double(ctx->ctl.B());
-    KernelFn fn = asp_kernel(grad_dtype);
-    LaunchShape &shape = ctx->asp_shape[grad_dtype];
-    rc = shape_for(ctx, fn, shape);
+    const bool wide = all_aligned32(buckets, n_buckets, worker, worker + 1);
+    const KernelInfo ki = asp_kernel(grad_dtype, wide);
+    LaunchShape &shape = ctx->asp_shape[grad_dtype][wide];
+    rc = shape_for(ctx, ki, shape);
     if (rc != OMNI_OK) return rc;
-    const unsigned long long tile = asp_tile_elems(grad_dtype);
+    const unsigned long long tile = ki.tile;
 
     AspParams p;
     int i = 0;
@@ -384,7 +417,7 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
         p.nb = nb;
         p.tiles = tiles;
         const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
-        rc = launch(ctx, fn, grid, &p, static_cast<cudaStream_t>(stream));
+        rc = launch(ctx, ki, grid, &p, static_cast<cudaStream_t>(stream));
         if (rc != OMNI_OK) return rc;
     }
     ctx->tally.arrivals += 1;
@@ -415,8 +448,8 @@ int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *gri
     if (grad_dtype != OMNI_F32 && grad_dtype != OMNI_BF16) return OMNI_ERR_BAD_CONFIG;
     int rc = ensure_device(ctx);
     if (rc != OMNI_OK) return rc;
-    LaunchShape &shape = ctx->bsp_shape[grad_dtype][K];
-    rc = shape_for(ctx, bsp_kernel(grad_dtype, K), shape);
+    LaunchShape &shape = ctx->bsp_shape[grad_dtype][1][K];
+    rc = shape_for(ctx, bsp_kernel(grad_dtype, K, true), shape);
     if (rc != OMNI_OK) return rc;
     *grid = shape.grid;
     *block = shape.block;

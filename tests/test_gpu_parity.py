@@ -164,6 +164,40 @@ def test_bsp_many_buckets_empty_and_ragged(kind):
     assert abs(o.stats().grad_sqnorm - sq_total) <= SQNORM_RTOL * sq_total
 
 
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+@pytest.mark.parametrize("K", [1, 4, 16, 32])
+def test_buffers_aligned_to_16_bytes_only(K, kind):
+    """Buffers that sit on a 16-byte but not a 32-byte boundary take the 128-bit kernels; one
+    misaligned buffer among aligned ones is enough.  Same results as the oracle, bit for bit."""
+    n = 5 * 8192 + 29
+    for which in ("all", "one_grad", "theta"):
+        theta, v, grads, plp = _make(K, n + 8, kind, 31 * K, lp=True)
+        sh = lambda buf, on: buf.t[(8 if buf.dtype == torch.bfloat16 else 4):][:n] if on else buf.t[:n]
+        th_t = sh(theta, which in ("all", "theta"))
+        v_t = sh(v, which == "all")
+        lp_t = sh(plp, which == "all")
+        g_t = [sh(g, which == "all" or (which == "one_grad" and k == K - 1)) for k, g in enumerate(grads)]
+        assert th_t.data_ptr() % 32 == (16 if which != "one_grad" else 0)
+        b = _random_batches(K, 32, K)
+        o = B.Omni(K, 32 * K, 1, 32 * K, 0.1)
+        bs = B.BucketSet([th_t], [g_t], [v_t], [lp_t])
+        th_o, v_o, g_np = to_np(th_t), to_np(v_t), [to_np(g) for g in g_t]
+        lp_o = np.zeros(n, np.uint16)
+        for _ in range(2):
+            o.aggregate_bsp(bs, b, 0.1, 0.9, 1e-4)
+            sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 1e-4, theta_lp=lp_o)
+        assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+        assert np.array_equal(to_np(th_t), th_o) and np.array_equal(to_np(v_t), v_o)
+        assert np.array_equal(to_np(lp_t), lp_o)
+        a = B.Omni(K, 32 * K, 1, 32 * K, 0.1, 1.0, B.ASP)
+        a.apply_asp(bs, K - 1, 17, 2, 0.1, 0.9, 1e-4)
+        O.asp_apply_f32(g_np[K - 1], 17, 32 * K, th_o, v_o, 0.1, 0.9, 1e-4, theta_lp=lp_o)
+        assert np.array_equal(to_np(th_t), th_o) and np.array_equal(to_np(v_t), v_o)
+        assert np.array_equal(to_np(lp_t), lp_o)
+        for buf in (theta, v, plp, *grads):
+            assert buf.intact()
+
+
 def test_empty_call_reads_zero_norm():
     o = B.Omni(2, 64, 4, 96, 0.1)
     theta, v, grads, _ = _make(2, 1000, "f32", 1)
