@@ -65,17 +65,31 @@ struct AspParams {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Launch shape per (gradient type, K): threads per CTA and gradient vectors per thread and
-// stream.  Chosen from timing sweeps on B200; the rule keeps roughly 0.4-0.6 KB of loads per
-// thread in flight.
+// Launch shape per (gradient type, K): threads per CTA, gradient vectors per thread and stream,
+// and CTAs per SM of the persistent grid.  Taken from timing scans on B200 over
+// threads x vectors x CTAs/SM: bandwidth peaks at a moderate number of resident threads
+// (about 500-770 thread-vectors per SM) and falls on both sides -- too few leave HBM latency
+// uncovered, too many widen the window of DRAM pages open at once.
 // ---------------------------------------------------------------------------------------------
-template <typename G> __host__ __device__ constexpr int bsp_threads(int K)
+struct Shape { int threads, chunks, ctas_per_sm; };
+
+template <typename G> __host__ __device__ constexpr Shape bsp_shape(int K)
 {
-    return sizeof(G) == 2 && K >= 12 ? 192 : 256;
+    if (sizeof(G) == 4) {
+        if (K >= 20) return {256, 1, 3};
+        if (K >= 11) return {192, 1, 3};
+        if (K >= 7) return {128, 2, 2};
+        if (K >= 3) return {128, 2, 3};
+        if (K == 2) return {128, 4, 1};
+        return {256, 2, 1};
+    }
+    if (K >= 12) return {192, 1, 3};
+    if (K >= 5) return {128, 2, 1};
+    return {192, 1, 3};
 }
-template <typename G> __host__ __device__ constexpr int bsp_chunks(int K) { return K <= 2 ? 4 : K <= 10 ? 2 : 1; }
 constexpr int kAspThreads = 256;
 constexpr int kAspChunks = 2;
+__host__ __device__ constexpr int asp_ctas_per_sm(bool momentum) { return momentum ? 1 : 2; }
 
 // ---------------------------------------------------------------------------------------------
 // 128- and 256-bit global memory access with streaming hints
@@ -293,18 +307,52 @@ __global__ void __launch_bounds__(THREADS) bsp_fused_kernel(const __grid_constan
                 if (has_lp) store_lp<Ge::LW>(bd.lp + off, th[c]);
             }
         } else {
-            // ragged last tile of a bucket: element by element, same arithmetic
-            for (unsigned long long j = base + tid; j < bd.n; j += THREADS) {
-                float acc = 0.0f;
+            // ragged last tile of a bucket: whole vectors as above (one chunk at a time), then the
+            // last partial vector element by element; same arithmetic
+#pragma unroll 1
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                if (off + E <= bd.n) {
+                    Raw<Ge::GW> raw[K];
+                    float th[E], vv[E], acc[E];
 #pragma unroll
-                for (int k = 0; k < K; ++k)
-                    acc = __fmaf_rn(p.lam[k], widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
-                float vj = mu != 0.0f ? __ldcs(bd.v + j) : 0.0f;
-                const float t = update_one(acc, __ldcs(bd.theta + j), vj, lr, mu, wd);
-                sq += (double)(acc * acc);
-                bd.theta[j] = t;
-                if (has_v) bd.v[j] = vj;
-                if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                    for (int k = 0; k < K; ++k) raw[k] = ld_ro<Ge::GW>(static_cast<const G *>(p.g[bi][k]) + off);
+                    load_floats<Ge::FW, Ge::FN>(bd.theta + off, th);
+                    if (mu != 0.0f) load_floats<Ge::FW, Ge::FN>(bd.v + off, vv);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[e] = 0.0f;
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        float gk[E];
+                        widen<G, Ge::GW>(raw[k], gk);
+                        const float lam = p.lam[k];
+#pragma unroll
+                        for (int e = 0; e < E; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
+                    }
+                    float part = 0.0f;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        part = __fmaf_rn(acc[e], acc[e], part);
+                        th[e] = update_one(acc[e], th[e], vv[e], lr, mu, wd);
+                    }
+                    sq += (double)part;
+                    store_floats<Ge::FW, Ge::FN>(bd.theta + off, th);
+                    if (has_v) store_floats<Ge::FW, Ge::FN>(bd.v + off, vv);
+                    if (has_lp) store_lp<Ge::LW>(bd.lp + off, th);
+                } else {
+                    for (unsigned long long j = off; j < bd.n; ++j) {
+                        float acc = 0.0f;
+#pragma unroll
+                        for (int k = 0; k < K; ++k)
+                            acc = __fmaf_rn(p.lam[k], widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
+                        float vj = mu != 0.0f ? __ldcs(bd.v + j) : 0.0f;
+                        const float t = update_one(acc, __ldcs(bd.theta + j), vj, lr, mu, wd);
+                        sq += (double)(acc * acc);
+                        bd.theta[j] = t;
+                        if (has_v) bd.v[j] = vj;
+                        if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                    }
+                }
             }
         }
     }
@@ -352,12 +400,30 @@ __global__ void __launch_bounds__(THREADS) asp_apply_kernel(const __grid_constan
                 if (has_lp) store_lp<Ge::LW>(bd.lp + off, th[c]);
             }
         } else {
-            for (unsigned long long j = base + tid; j < bd.n; j += THREADS) {
-                float vj = mu != 0.0f ? __ldcs(bd.v + j) : 0.0f;
-                const float t = update_one(widen1<G>(g, j), __ldcs(bd.theta + j), vj, eta, mu, wd);
-                bd.theta[j] = t;
-                if (has_v) bd.v[j] = vj;
-                if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+            // ragged last tile: whole vectors one chunk at a time, then the partial vector
+#pragma unroll 1
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                if (off + E <= bd.n) {
+                    float th[E], vv[E], gk[E];
+                    const Raw<Ge::GW> raw = ld_ro<Ge::GW>(g + off);
+                    load_floats<Ge::FW, Ge::FN>(bd.theta + off, th);
+                    if (mu != 0.0f) load_floats<Ge::FW, Ge::FN>(bd.v + off, vv);
+                    widen<G, Ge::GW>(raw, gk);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) th[e] = update_one(gk[e], th[e], vv[e], eta, mu, wd);
+                    store_floats<Ge::FW, Ge::FN>(bd.theta + off, th);
+                    if (has_v) store_floats<Ge::FW, Ge::FN>(bd.v + off, vv);
+                    if (has_lp) store_lp<Ge::LW>(bd.lp + off, th);
+                } else {
+                    for (unsigned long long j = off; j < bd.n; ++j) {
+                        float vj = mu != 0.0f ? __ldcs(bd.v + j) : 0.0f;
+                        const float t = update_one(widen1<G>(g, j), __ldcs(bd.theta + j), vj, eta, mu, wd);
+                        bd.theta[j] = t;
+                        if (has_v) bd.v[j] = vj;
+                        if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                    }
+                }
             }
         }
     }

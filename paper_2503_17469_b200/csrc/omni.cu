@@ -16,6 +16,7 @@ using KernelFn = const void *;
 struct KernelInfo {
     KernelFn fn = nullptr;
     int threads = 0;
+    int ctas_per_sm = 0;          // wanted CTAs per SM (capped by what fits)
     unsigned long long tile = 0;  // elements per tile
 };
 
@@ -34,7 +35,7 @@ struct omni_ctx {
     int last_cuda = 0;
     uint64_t launches = 0;
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
-    omni::LaunchShape asp_shape[2][2];                  // [dtype][wide]
+    omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
 };
 
 namespace omni {
@@ -51,9 +52,9 @@ namespace {
 
 template <typename G, int K, bool WIDE> KernelInfo bsp_info()
 {
-    constexpr int T = bsp_threads<G>(K), C = bsp_chunks<G>(K);
-    return {reinterpret_cast<KernelFn>(&bsp_fused_kernel<G, K, T, C, WIDE>), T,
-            (unsigned long long)T * Geo<G, WIDE>::E * C};
+    constexpr Shape sh = bsp_shape<G>(K);
+    return {reinterpret_cast<KernelFn>(&bsp_fused_kernel<G, K, sh.threads, sh.chunks, WIDE>), sh.threads,
+            sh.ctas_per_sm, (unsigned long long)sh.threads * Geo<G, WIDE>::E * sh.chunks};
 }
 
 template <typename G, bool WIDE> KernelInfo bsp_kernel_for(int K)
@@ -75,15 +76,15 @@ KernelInfo bsp_kernel(int dtype, int K, bool wide)
     return wide ? bsp_kernel_for<float, true>(K) : bsp_kernel_for<float, false>(K);
 }
 
-template <typename G, bool WIDE> KernelInfo asp_info()
+template <typename G, bool WIDE> KernelInfo asp_info(bool momentum)
 {
     return {reinterpret_cast<KernelFn>(&asp_apply_kernel<G, kAspThreads, kAspChunks, WIDE>), kAspThreads,
-            (unsigned long long)kAspThreads * Geo<G, WIDE>::E * kAspChunks};
+            asp_ctas_per_sm(momentum), (unsigned long long)kAspThreads * Geo<G, WIDE>::E * kAspChunks};
 }
-KernelInfo asp_kernel(int dtype, bool wide)
+KernelInfo asp_kernel(int dtype, bool wide, bool momentum)
 {
-    if (dtype == OMNI_BF16) return wide ? asp_info<__nv_bfloat16, true>() : asp_info<__nv_bfloat16, false>();
-    return wide ? asp_info<float, true>() : asp_info<float, false>();
+    if (dtype == OMNI_BF16) return wide ? asp_info<__nv_bfloat16, true>(momentum) : asp_info<__nv_bfloat16, false>(momentum);
+    return wide ? asp_info<float, true>(momentum) : asp_info<float, false>(momentum);
 }
 
 // First kernel-launching call of a context: bind to the current device, allocate the workspace.
@@ -113,13 +114,15 @@ int ensure_device(omni_ctx *ctx)
     return OMNI_OK;
 }
 
-// Persistent grid = SM count x resident CTAs per SM of that kernel, capped by the slot count.
+// Persistent grid = SM count x CTAs per SM (the kernel's tuned figure, capped by what is resident
+// at once and by the partial-sum slots).
 int shape_for(omni_ctx *ctx, const KernelInfo &ki, LaunchShape &s)
 {
     if (s.grid > 0) return OMNI_OK;
     int per_sm = 0;
     OMNI_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ki.fn, ki.threads, 0));
     if (per_sm < 1) per_sm = 1;
+    if (ki.ctas_per_sm > 0 && per_sm > ki.ctas_per_sm) per_sm = ki.ctas_per_sm;
     int grid = ctx->sm_count * per_sm;
     if (grid > kMaxGrid) grid = kMaxGrid / ctx->sm_count * ctx->sm_count;
     s.grid = grid;
@@ -391,8 +394,8 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
                              ? double(lr)
                              : double(lr) * double(b_used) / double(ctx->ctl.B());
     const bool wide = all_aligned32(buckets, n_buckets, worker, worker + 1);
-    const KernelInfo ki = asp_kernel(grad_dtype, wide);
-    LaunchShape &shape = ctx->asp_shape[grad_dtype][wide];
+    const KernelInfo ki = asp_kernel(grad_dtype, wide, momentum != 0.0f);
+    LaunchShape &shape = ctx->asp_shape[grad_dtype][wide][momentum != 0.0f];
     rc = shape_for(ctx, ki, shape);
     if (rc != OMNI_OK) return rc;
     const unsigned long long tile = ki.tile;
