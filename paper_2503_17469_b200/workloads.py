@@ -275,22 +275,24 @@ def make_buffers(cfg: Config, device, gen: Optional[torch.Generator] = None, n_g
     lay = cfg.layout()
     K = cfg.K if n_grads is None else n_grads
     gdt = torch.bfloat16 if cfg.grad_dtype == "bf16" else torch.float32
-    theta = torch.zeros(lay.total, dtype=torch.float32, device=device)
-    v = torch.zeros(lay.total, dtype=torch.float32, device=device)
-    grads = [torch.zeros(lay.total, dtype=gdt, device=device) for _ in range(K)]
     n_t = len(cfg.shapes)
     if cfg.grad_std is None:
         e = torch.rand(n_t, generator=gen, dtype=torch.float64, device=device).cpu()
         stds = [float(10.0 ** (-5.0 + 3.0 * x)) for x in e.tolist()]
     else:
         stds = [cfg.grad_std] * n_t
+    # per-element standard deviation of the gradient; zero on padding
+    std_vec = torch.zeros(lay.total, dtype=torch.float32, device=device)
     for ti, start, ne in lay.tensor_slices():
-        theta[start:start + ne].normal_(0.0, cfg.param_std, generator=gen)
-    for g in grads:
-        for ti, start, ne in lay.tensor_slices():
-            if gdt == torch.float32:
-                g[start:start + ne].normal_(0.0, stds[ti], generator=gen)
-            else:
-                tmp = torch.empty(ne, dtype=torch.float32, device=device).normal_(0.0, stds[ti], generator=gen)
-                g[start:start + ne].copy_(tmp)
+        std_vec[start:start + ne] = stds[ti]
+    real = std_vec > 0
+    theta = torch.empty(lay.total, dtype=torch.float32, device=device).normal_(0.0, cfg.param_std, generator=gen)
+    theta.mul_(real)
+    v = torch.zeros(lay.total, dtype=torch.float32, device=device)
+    grads = []
+    for _ in range(K):
+        g = torch.empty(lay.total, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
+        g.mul_(std_vec)
+        grads.append(g if gdt == torch.float32 else g.to(gdt))
+    del std_vec, real
     return Buffers(layout=lay, theta=theta, v=v, grads=grads, grad_std=stds)
