@@ -285,14 +285,14 @@ def make_buffers(cfg: Config, device, gen: Optional[torch.Generator] = None, n_g
     std_vec = torch.zeros(lay.total, dtype=torch.float32, device=device)
     for ti, start, ne in lay.tensor_slices():
         std_vec[start:start + ne] = stds[ti]
-    real = std_vec > 0
+    pad = std_vec == 0          # padding stays exactly +0 in every buffer
     theta = torch.empty(lay.total, dtype=torch.float32, device=device).normal_(0.0, cfg.param_std, generator=gen)
-    theta.mul_(real)
+    theta.masked_fill_(pad, 0.0)
     v = torch.zeros(lay.total, dtype=torch.float32, device=device)
     grads = []
     for _ in range(K):
         g = torch.empty(lay.total, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
-        g.mul_(std_vec)
+        g.mul_(std_vec).masked_fill_(pad, 0.0)
         grads.append(g if gdt == torch.float32 else g.to(gdt))
-    del std_vec, real
+    del std_vec, pad
     return Buffers(layout=lay, theta=theta, v=v, grads=grads, grad_std=stds)
