@@ -164,6 +164,41 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
                             const void *const *host_grads, const int32_t *b, float lr, float momentum,
                             float weight_decay, void *stream, double *grad_sqnorm);
 
+/* The same fused step as omni_aggregate_bsp for callers that are not allowed to allocate device
+ * memory when they run a step.  (The paper has no counterpart: this is a deployment variant of
+ * the call above, not part of the method.)
+ *
+ * Who needs it: code that runs inside another framework's allocator callback or under its
+ * allocator lock, processes whose device memory has all been handed to a pool at start-up, and
+ * latency-critical loops that ban calls which may synchronise the device, as cudaMalloc and
+ * cudaFree may.  omni_aggregate_bsp allocates a small workspace on a context's first launch;
+ * this function calls no cudaMalloc, cudaFree or any allocating routine, ever.  Its kernel's
+ * scratch (per-CTA partial sums, the norm cell and a ticket counter, about 19 KB) is a fixed
+ * array inside the library's device image: every GPU that loads the library holds it until the
+ * process exits.
+ *
+ * It takes no context: K, the batches and the flags (OMNI_UNSCALED_MEAN) come as arguments and
+ * lambda_k = b_k / sum b.  Arithmetic, layouts and alignment rules are those of
+ * omni_aggregate_bsp.  grad_sqnorm_dev (DEVICE pointer, 8-byte aligned, may be NULL) receives
+ * the squared norm of the aggregate by a copy enqueued after the kernel.  Enqueues on `stream`,
+ * does not synchronise.
+ *
+ * Limits: at most OMNI_NOALLOC_MAX_BUCKETS non-empty buckets and OMNI_NOALLOC_MAX_ELEMENTS
+ * elements in total; more returns OMNI_ERR_TOO_LARGE and does nothing.
+ * Sharing: all calls on one device use the same array, which keeps the previous call's
+ * contents; the function zeroes the cells that must start at zero before each launch.  Calls
+ * whose kernels overlap on the GPU (issued on different streams without ordering) race on it
+ * and give wrong norms: keep them on one stream or order them with events.
+ * First call: the first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) with that device current; make that call before any stream capture.
+ * It is not thread-safe against another first call on the same device.
+ * Errors: BAD_K, NULL, BAD_CONFIG, BAD_BATCH (some b_k < 1), ALIGN, TOO_LARGE, CUDA. */
+#define OMNI_NOALLOC_MAX_BUCKETS 8
+#define OMNI_NOALLOC_MAX_ELEMENTS (1ull << 31)
+int omni_aggregate_bsp_noalloc(int32_t K, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                               const int32_t *b, uint32_t flags, float lr, float momentum, float weight_decay,
+                               double *grad_sqnorm_dev, void *stream);
+
 /* Synchronises `stream` and fills *out (host). */
 int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream);
 

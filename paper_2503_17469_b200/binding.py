@@ -26,8 +26,10 @@ EXPORTS = (
     "omni_strerror", "omni_create", "omni_destroy", "omni_get_batches", "omni_set_batches",
     "omni_rebatch", "omni_asp_report", "omni_rebatch_static", "omni_aggregate_bsp",
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
-    "omni_query_launch", "omni_kernel_launches",
+    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc",
 )
+NOALLOC_MAX_BUCKETS = 8
+NOALLOC_MAX_ELEMENTS = 1 << 31
 
 
 class omni_config(C.Structure):
@@ -74,6 +76,8 @@ def lib() -> C.CDLL:
     L.omni_query_launch.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
     L.omni_kernel_launches.argtypes = [vp]
     L.omni_kernel_launches.restype = C.c_uint64
+    L.omni_aggregate_bsp_noalloc.argtypes = [i32, C.POINTER(omni_bucket), i32, i32, C.POINTER(i32), C.c_uint32,
+                                             f32, f32, f32, vp, vp]
     _lib = L
     return L
 
@@ -151,6 +155,25 @@ class BucketSet:
         return cls([theta[s] for s in sl], [[g[s] for g in grads] for s in sl],
                    [v[s] for s in sl] if v is not None else None,
                    [theta_lp[s] for s in sl] if theta_lp is not None else None)
+
+
+def aggregate_bsp_noalloc(buckets: "BucketSet", b: Sequence[int], lr: float, momentum: float = 0.0,
+                          weight_decay: float = 0.0, flags: int = 0, grad_sqnorm_out=None, stream=None) -> None:
+    """The fused synchronous step through ``omni_aggregate_bsp_noalloc``, the entry point for
+    callers that may not allocate device memory while stepping (allocator callbacks, processes
+    whose memory is all pooled, loops that ban device-synchronising calls).  No context: K is
+    ``buckets.K``.  ``grad_sqnorm_out``: optional one-element float64 CUDA tensor that receives
+    the squared norm.  Calls on one device share a fixed scratch array: keep them ordered on a
+    stream, and make the first call on a device outside stream capture."""
+    K = buckets.K
+    ptr = None
+    if grad_sqnorm_out is not None:
+        assert grad_sqnorm_out.numel() == 1 and grad_sqnorm_out.element_size() == 8 and grad_sqnorm_out.is_cuda
+        ptr = C.c_void_p(grad_sqnorm_out.data_ptr())
+    rc = lib().omni_aggregate_bsp_noalloc(K, buckets.array, buckets.n_buckets, buckets.dtype, (C.c_int32 * K)(*b),
+                                          flags, lr, momentum, weight_decay, ptr, Omni._stream(stream))
+    if rc != OK:
+        raise OmniError(rc)
 
 
 class Omni:

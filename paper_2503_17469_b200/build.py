@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libomni.so"
-SOURCES = [CSRC / "omni.cu", CSRC / "controller.cpp"]
+SOURCES = [CSRC / "omni.cu", CSRC / "noalloc.cu", CSRC / "controller.cpp"]
 HEADERS = [CSRC / "kernels.cuh", CSRC / "controller.h", PKG.parent / "include" / "omni.h"]
 
 NVCC_FLAGS = [
