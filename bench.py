@@ -194,13 +194,13 @@ def bsp_line(job, ms, steps, launches, peak):
 # --------------------------------------------------------------------------------------------
 # CPU oracle legs
 # --------------------------------------------------------------------------------------------
-def oracle_sample(name, target_s, torch, W):
-    """Times the single-threaded oracle on a prefix of the configuration's first bucket."""
+def oracle_sample(name, n_max, torch, W):
+    """The single-threaded oracle on a prefix (at most n_max elements) of the configuration's first bucket."""
     from oracle import oracle as O
     import numpy as np
 
     cfg = W.config(name)
-    n = min(cfg.layout().buckets[0].n, 4_000_000)
+    n = int(min(cfg.layout().buckets[0].n, n_max))
     gen = torch.Generator().manual_seed(cfg.seed)
     gdt = torch.bfloat16 if cfg.grad_dtype == "bf16" else torch.float32
     g = []
@@ -220,7 +220,7 @@ def oracle_sample(name, target_s, torch, W):
 
 
 def cpu_baseline(name, target_s, torch, W):
-    n, step = oracle_sample(name, target_s, torch, W)
+    n, step = oracle_sample(name, 4_000_000, torch, W)
     step(0)
     t0 = time.perf_counter()
     step(1)
@@ -240,7 +240,14 @@ def reference_arm(args, torch, W):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n, step = oracle_sample(HEADLINE, 0, torch, W)
+    # size the per-step sample so that warm-up + steps take about two minutes of CPU time
+    n_cal, cal = oracle_sample(HEADLINE, 262_144, torch, W)
+    cal(0)
+    t0 = time.perf_counter()
+    cal(1)
+    per_elem = (time.perf_counter() - t0) / n_cal
+    budget = 120.0 / (args.steps + args.warmup) / per_elem
+    n, step = oracle_sample(HEADLINE, max(65_536, min(4_000_000, budget)), torch, W)
     cfg = W.config(HEADLINE)
     for i in range(args.warmup):
         step(i)
@@ -260,6 +267,47 @@ def reference_arm(args, torch, W):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
+
+
+class Ranks:
+    """One process per GPU, no data exchange between them (independent replicas).  The only
+    cross-rank traffic is the timing protocol: a barrier on both sides of the timed region and a
+    MAX reduction of the per-rank times.  backend "nccl" on GPUs; "gloo" lets the CPU tests run
+    the same protocol."""
+
+    def __init__(self, backend="nccl", device=None):
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.dist = None
+        self.device = device
+        if self.world > 1:
+            import torch.distributed as dist
+
+            kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
+            dist.init_process_group(backend, **kw)
+            self.dist = dist
+
+    def barrier(self):
+        if self.dist:
+            self.dist.barrier()
+
+    def max_over_ranks(self, x: float) -> float:
+        if not self.dist:
+            return x
+        import torch
+
+        t = torch.tensor([x], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def whole_job_value(self, units_per_rank: float, ms_local: float) -> float:
+        """Units all ranks processed divided by the slowest rank's time."""
+        return self.world * units_per_rank / (self.max_over_ranks(ms_local) * 1e-3)
+
+    def close(self):
+        if self.dist:
+            self.dist.destroy_process_group()
 
 
 # --------------------------------------------------------------------------------------------
@@ -288,27 +336,16 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     B.lib()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ranks = Ranks("nccl", torch.device("cuda", local))
+    rank, world, dist = ranks.rank, ranks.world, ranks.dist
 
     def barrier():
-        if dist:
-            dist.barrier()
+        ranks.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if not dist:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    max_over_ranks = ranks.max_over_ranks
 
     peak, peak_kind = measured_peak()
     job = BspJob(HEADLINE, torch, W, B)
@@ -373,8 +410,7 @@ def main():
             "extras": extras,
         }
         print(json.dumps(line))
-    if dist:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 def run_extras(torch, W, B, peak, headline_job):
