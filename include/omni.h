@@ -153,6 +153,18 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
                    int32_t worker, int32_t b_used, int32_t tau, float lr, float momentum, float weight_decay,
                    void *stream);
 
+/* A batch of m queued asynchronous arrivals applied in one pass over the parameters, in the order
+ * given: exactly the result of m successive omni_apply_asp calls (the element goes through the
+ * m updates of Eq. 5b one after the other, theta and v staying in registers), but theta and v
+ * are read and written once, so the traffic is 4m+8 (+8 with momentum) bytes per parameter
+ * instead of 12m (20m).  workers[m], b_used[m], tau[m]: host arrays; a worker may appear more
+ * than once (its buffer is then applied again).  1 <= m <= OMNI_MAX_ASP_BATCH.
+ * Errors: as omni_apply_asp, plus TOO_LARGE for m out of range. */
+#define OMNI_MAX_ASP_BATCH 16
+int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype, int32_t m,
+                         const int32_t *workers, const int32_t *b_used, const int32_t *tau, float lr, float momentum,
+                         float weight_decay, void *stream);
+
 /* Same step as omni_aggregate_bsp for gradients that arrive in HOST memory (pinned memory gives
  * asynchronous copies).  host_grads: host array of n_buckets*K host pointers, entry [i*K + k] =
  * worker k's gradient for bucket i.  buckets[i].grads must point at K device staging buffers of

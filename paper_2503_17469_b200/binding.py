@@ -26,8 +26,9 @@ EXPORTS = (
     "omni_strerror", "omni_create", "omni_destroy", "omni_get_batches", "omni_set_batches",
     "omni_rebatch", "omni_asp_report", "omni_rebatch_static", "omni_aggregate_bsp",
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
-    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc",
+    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch",
 )
+MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
 NOALLOC_MAX_ELEMENTS = 1 << 31
 
@@ -69,6 +70,8 @@ def lib() -> C.CDLL:
     L.omni_rebatch_static.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
     L.omni_aggregate_bsp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(i32), f32, f32, f32, vp]
     L.omni_apply_asp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, f32, f32, f32, vp]
+    L.omni_apply_asp_batch.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, C.POINTER(i32), C.POINTER(i32),
+                                       C.POINTER(i32), f32, f32, f32, vp]
     L.omni_aggregate_bsp_host.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(vp), C.POINTER(i32),
                                           f32, f32, f32, vp, C.POINTER(C.c_double)]
     L.omni_get_stats.argtypes = [vp, C.POINTER(omni_stats), vp]
@@ -261,6 +264,15 @@ class Omni:
                   weight_decay: float = 0.0, stream=None) -> None:
         self._check(lib().omni_apply_asp(self._h, buckets.array, buckets.n_buckets, buckets.dtype, worker, b_used,
                                          tau, lr, momentum, weight_decay, self._stream(stream)))
+
+    def apply_asp_batch(self, buckets: BucketSet, workers: Sequence[int], b_used: Sequence[int], tau: Sequence[int],
+                        lr: float, momentum: float = 0.0, weight_decay: float = 0.0, stream=None) -> None:
+        """m queued arrivals in one pass (same result as m ``apply_asp`` calls in that order)."""
+        m = len(workers)
+        arr = C.c_int32 * m
+        self._check(lib().omni_apply_asp_batch(self._h, buckets.array, buckets.n_buckets, buckets.dtype, m,
+                                               arr(*workers), arr(*b_used), arr(*tau), lr, momentum, weight_decay,
+                                               self._stream(stream)))
 
     def stats(self, stream=None) -> Stats:
         s = omni_stats()

@@ -28,13 +28,26 @@ def stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> Path:
+    """Compile every source to an object (in parallel), then link the shared library."""
     if not (force or stale()):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    objdir = PKG / "_build"
+    objdir.mkdir(exist_ok=True)
+    compile_flags = [f for f in NVCC_FLAGS if f != "-shared"] + (["-Xptxas", "-v"] if verbose else [])
+    jobs = []
+    for src in SOURCES:
+        obj = objdir / (src.stem + f".{os.getpid()}.o")
+        jobs.append((obj, subprocess.Popen([nvcc, *compile_flags, "-c", "-o", str(obj), str(src)])))
+    failed = [str(o) for o, p in jobs if p.wait() != 0]
+    if failed:
+        raise RuntimeError(f"nvcc failed for {failed}")
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp), *map(str, SOURCES)]
-    subprocess.run(cmd, check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", str(tmp),
+                    *[str(o) for o, _ in jobs]], check=True)
     os.replace(tmp, LIB)
+    for o, _ in jobs:
+        o.unlink(missing_ok=True)
     return LIB
 
 

@@ -429,4 +429,92 @@ __global__ void __launch_bounds__(THREADS) asp_apply_kernel(const __grid_constan
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Batched asynchronous apply: M queued arrivals in one pass.  Same streaming skeleton as the
+// synchronous kernel (M gradient streams + theta + v), but instead of one weighted sum followed
+// by one update, each element goes through the M per-arrival updates in order with theta and v
+// held in registers: bit-identical to M single-arrival launches at 4M+8 (+8 with momentum)
+// bytes per parameter instead of 12M (20M).  p.lam[k] carries eta_k.  No norm is produced.
+// ---------------------------------------------------------------------------------------------
+template <typename G, int M, int THREADS, int C, bool WIDE>
+__global__ void __launch_bounds__(THREADS) asp_batch_kernel(const __grid_constant__ BspParams p)
+{
+    using Ge = Geo<G, WIDE>;
+    constexpr int E = Ge::E;
+    constexpr unsigned long long TILE = (unsigned long long)THREADS * E * C;
+    const int tid = threadIdx.x;
+    const float mu = p.mu, wd = p.wd;
+
+    for (unsigned long long tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
+        const int bi = find_bucket<kMaxBucketsPerLaunch>(p.bk, p.nb, tile);
+        const BucketDesc bd = p.bk[bi];
+        const unsigned long long base = (tile - bd.tile0) * TILE;
+        const bool has_v = bd.v != nullptr, has_lp = bd.lp != nullptr;
+
+        if (base + TILE <= bd.n) {
+            Raw<Ge::GW> raw[C][M];
+            float th[C][E], vv[C][E];
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+#pragma unroll
+                for (int k = 0; k < M; ++k) raw[c][k] = ld_ro<Ge::GW>(static_cast<const G *>(p.g[bi][k]) + off);
+                load_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (mu != 0.0f) load_floats<Ge::FW, Ge::FN>(bd.v + off, vv[c]);
+            }
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+#pragma unroll
+                for (int k = 0; k < M; ++k) {
+                    float gk[E];
+                    widen<G, Ge::GW>(raw[c][k], gk);
+                    const float eta = p.lam[k];
+#pragma unroll
+                    for (int e = 0; e < E; ++e) th[c][e] = update_one(gk[e], th[c][e], vv[c][e], eta, mu, wd);
+                }
+                store_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (has_v) store_floats<Ge::FW, Ge::FN>(bd.v + off, vv[c]);
+                if (has_lp) store_lp<Ge::LW>(bd.lp + off, th[c]);
+            }
+        } else {
+            // ragged last tile: whole vectors one chunk at a time, then the partial vector
+#pragma unroll 1
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                if (off + E <= bd.n) {
+                    Raw<Ge::GW> raw[M];
+                    float th[E], vv[E];
+#pragma unroll
+                    for (int k = 0; k < M; ++k) raw[k] = ld_ro<Ge::GW>(static_cast<const G *>(p.g[bi][k]) + off);
+                    load_floats<Ge::FW, Ge::FN>(bd.theta + off, th);
+                    if (mu != 0.0f) load_floats<Ge::FW, Ge::FN>(bd.v + off, vv);
+#pragma unroll
+                    for (int k = 0; k < M; ++k) {
+                        float gk[E];
+                        widen<G, Ge::GW>(raw[k], gk);
+                        const float eta = p.lam[k];
+#pragma unroll
+                        for (int e = 0; e < E; ++e) th[e] = update_one(gk[e], th[e], vv[e], eta, mu, wd);
+                    }
+                    store_floats<Ge::FW, Ge::FN>(bd.theta + off, th);
+                    if (has_v) store_floats<Ge::FW, Ge::FN>(bd.v + off, vv);
+                    if (has_lp) store_lp<Ge::LW>(bd.lp + off, th);
+                } else {
+                    for (unsigned long long j = off; j < bd.n; ++j) {
+                        float vj = mu != 0.0f ? __ldcs(bd.v + j) : 0.0f;
+                        float t = __ldcs(bd.theta + j);
+#pragma unroll
+                        for (int k = 0; k < M; ++k)
+                            t = update_one(widen1<G>(static_cast<const G *>(p.g[bi][k]), j), t, vj, p.lam[k], mu, wd);
+                        bd.theta[j] = t;
+                        if (has_v) bd.v[j] = vj;
+                        if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                    }
+                }
+            }
+        }
+    }
+}
+
 }  // namespace omni

@@ -36,6 +36,7 @@ struct omni_ctx {
     uint64_t launches = 0;
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
+    omni::LaunchShape seq_shape[2][2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][wide][M]
 };
 
 namespace omni {
@@ -74,6 +75,29 @@ KernelInfo bsp_kernel(int dtype, int K, bool wide)
 {
     if (dtype == OMNI_BF16) return wide ? bsp_kernel_for<__nv_bfloat16, true>(K) : bsp_kernel_for<__nv_bfloat16, false>(K);
     return wide ? bsp_kernel_for<float, true>(K) : bsp_kernel_for<float, false>(K);
+}
+
+// Batched asynchronous apply, M = arrivals in the batch; launch shape as the synchronous kernel with K = M.
+template <typename G, int M, bool WIDE> KernelInfo seq_info()
+{
+    constexpr Shape sh = bsp_shape<G>(M);
+    return {reinterpret_cast<KernelFn>(&asp_batch_kernel<G, M, sh.threads, sh.chunks, WIDE>), sh.threads,
+            sh.ctas_per_sm, (unsigned long long)sh.threads * Geo<G, WIDE>::E * sh.chunks};
+}
+template <typename G, bool WIDE> KernelInfo seq_kernel_for(int M)
+{
+    switch (M) {
+#define OMNI_CASE(k) case k: return seq_info<G, k, WIDE>();
+        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
+        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
+#undef OMNI_CASE
+    }
+    return {};
+}
+KernelInfo seq_kernel(int dtype, int M, bool wide)
+{
+    if (dtype == OMNI_BF16) return wide ? seq_kernel_for<__nv_bfloat16, true>(M) : seq_kernel_for<__nv_bfloat16, false>(M);
+    return wide ? seq_kernel_for<float, true>(M) : seq_kernel_for<float, false>(M);
 }
 
 template <typename G, bool WIDE> KernelInfo asp_info(bool momentum)
@@ -426,6 +450,68 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
     ctx->tally.arrivals += 1;
     ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
     if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+    return OMNI_OK;
+}
+
+int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype, int32_t m,
+                         const int32_t *workers, const int32_t *b_used, const int32_t *tau, float lr, float momentum,
+                         float weight_decay, void *stream)
+{
+    if (!ctx || !workers || !b_used || !tau) return OMNI_ERR_NULL;
+    if (m < 1 || m > OMNI_MAX_ASP_BATCH) return OMNI_ERR_TOO_LARGE;
+    const int K = ctx->ctl.K();
+    for (int i = 0; i < m; ++i) {
+        if (workers[i] < 0 || workers[i] >= K) return OMNI_ERR_BAD_WORKER;
+        if (b_used[i] < 1) return OMNI_ERR_BAD_BATCH;
+        if (tau[i] < 0) return OMNI_ERR_BAD_TAU;
+    }
+    int rc = OMNI_OK;
+    for (int i = 0; i < m && rc == OMNI_OK; ++i) rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, workers[i], momentum);
+    if (rc != OMNI_OK) return rc;
+    rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+
+    bool wide = true;
+    for (int i = 0; i < m; ++i) wide = wide && all_aligned32(buckets, n_buckets, workers[i], workers[i] + 1);
+    const KernelInfo ki = seq_kernel(grad_dtype, m, wide);
+    LaunchShape &shape = ctx->seq_shape[grad_dtype][wide][m];
+    rc = shape_for(ctx, ki, shape);
+    if (rc != OMNI_OK) return rc;
+
+    BspParams p;
+    int i = 0;
+    while (i < n_buckets) {
+        std::memset(&p, 0, sizeof p);
+        unsigned long long tiles = 0;
+        int nb = 0;
+        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+            const omni_bucket &bk = buckets[i];
+            if (bk.n == 0) continue;
+            p.bk[nb] = {static_cast<float *>(bk.param), static_cast<float *>(bk.momentum),
+                        static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
+            for (int a = 0; a < m; ++a) p.g[nb][a] = bk.grads[workers[a]];
+            tiles += (bk.n + ki.tile - 1) / ki.tile;
+            ++nb;
+        }
+        if (nb == 0) break;
+        // Eq. 5b per arrival: eta = lr * b_used / B, in double, rounded once to float
+        for (int a = 0; a < m; ++a)
+            p.lam[a] = float((ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
+                                 ? double(lr)
+                                 : double(lr) * double(b_used[a]) / double(ctx->ctl.B()));
+        p.mu = momentum; p.wd = weight_decay;
+        p.nb = nb;
+        p.tiles = tiles;
+        p.ws = ctx->ws;
+        const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
+        rc = launch(ctx, ki, grid, &p, static_cast<cudaStream_t>(stream));
+        if (rc != OMNI_OK) return rc;
+    }
+    for (int a = 0; a < m; ++a) {
+        ctx->tally.arrivals += 1;
+        ctx->tally.tau_hist[tau[a] < OMNI_TAU_BINS - 1 ? tau[a] : OMNI_TAU_BINS - 1] += 1;
+        if (tau[a] > ctx->tally.tau_max) ctx->tally.tau_max = tau[a];
+    }
     return OMNI_OK;
 }
 

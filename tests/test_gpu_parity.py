@@ -1,5 +1,6 @@
 """GPU parity: the CUDA library, called through its C ABI, against the CPU oracle, element by
 element on the same seeded inputs."""
+import ctypes as C
 import math
 
 import numpy as np
@@ -271,6 +272,44 @@ def test_asp_parity_over_sizes(kind, mu, wd):
         for t in taus:
             ref.record(t)
         assert st.arrivals == 4 and st.tau_hist == ref.hist.tolist() and st.tau_max == ref.tau_max
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+@pytest.mark.parametrize("mu,wd", [(0.0, 0.0), (0.9, 1e-4)])
+def test_asp_batched_apply_equals_successive_arrivals(kind, mu, wd):
+    """m queued arrivals in one pass give the bits of m single-arrival updates in that order
+    (oracle: m successive applications of the per-arrival rule), for several m and ragged sizes."""
+    K = 6
+    rng = np.random.default_rng(17)
+    for m, n in [(1, 4097), (2, 100_003), (3, 7), (5, 3 * 8192 + 17), (16, 60_001)]:
+        theta, v, grads, plp = _make(K, n, kind, 3000 + m, lp=True, momentum=mu != 0)
+        o = B.Omni(K, 192, 4, 96, 0.1, 1.0, B.ASP)
+        bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t] if v else None, [plp.t])
+        workers = [int(x) for x in rng.integers(0, K, m)]
+        b_used = [int(x) for x in rng.integers(4, 97, m)]
+        taus = [int(x) for x in rng.integers(0, 50, m)]
+        th_o = to_np(theta.t)
+        v_o = to_np(v.t) if v else None
+        lp_o = np.zeros(n, np.uint16)
+        g_np = [to_np(g.t) for g in grads]
+        o.apply_asp_batch(bs, workers, b_used, taus, 0.1, mu, wd)
+        ref = O.TauStats()
+        for k, bu, tau in zip(workers, b_used, taus):
+            O.asp_apply_f32(g_np[k], bu, 192, th_o, v_o, 0.1, mu, wd, theta_lp=lp_o)
+            ref.record(tau)
+        assert np.array_equal(to_np(theta.t), th_o), (m, n)
+        if v:
+            assert np.array_equal(to_np(v.t), v_o)
+        assert np.array_equal(to_np(plp.t), lp_o)
+        st = o.stats()
+        assert st.arrivals == m and st.tau_hist == ref.hist.tolist() and st.tau_max == ref.tau_max
+        assert theta.intact() and plp.intact() and all(g.intact() for g in grads)
+    L, h = B.lib(), o._h
+    i32 = lambda *a: (C.c_int32 * len(a))(*a)
+    assert L.omni_apply_asp_batch(h, bs.array, 1, bs.dtype, 17, i32(*[0] * 17), i32(*[8] * 17), i32(*[0] * 17), 0.1, mu, wd, None) == B.ERR_TOO_LARGE
+    assert L.omni_apply_asp_batch(h, bs.array, 1, bs.dtype, 2, i32(0, K), i32(8, 8), i32(0, 0), 0.1, mu, wd, None) == B.ERR_BAD_WORKER
+    assert L.omni_apply_asp_batch(h, bs.array, 1, bs.dtype, 2, i32(0, 1), i32(8, 0), i32(0, 0), 0.1, mu, wd, None) == B.ERR_BAD_BATCH
+    assert L.omni_apply_asp_batch(h, bs.array, 1, bs.dtype, 2, i32(0, 1), i32(8, 8), i32(0, -1), 0.1, mu, wd, None) == B.ERR_BAD_TAU
 
 
 def test_asp_no_lr_scale_flag():
