@@ -144,13 +144,13 @@ def throughput_schedule(cfg, n, W, torch):
 class BspJob:
     """Buffers + context of one synchronous configuration on the current device."""
 
-    def __init__(self, name, torch, W, B, with_lp=False):
+    def __init__(self, name, torch, W, B, with_lp=False, flags=0):
         self.cfg = cfg = W.config(name)
         self.torch = torch
         self.buf = W.make_buffers(cfg, torch.device("cuda", torch.cuda.current_device()))
         lay = self.buf.layout
         self.theta_lp = torch.zeros(lay.total, dtype=torch.bfloat16, device=self.buf.theta.device) if with_lp else None
-        self.omni = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.BSP)
+        self.omni = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.BSP, flags)
         self.buckets = B.BucketSet.from_flat(lay, self.buf.theta, self.buf.grads, self.buf.v, self.theta_lp)
         self.bytes_per_step = cfg.bytes_per_param(with_lp) * cfg.P
         self.W = W
@@ -418,12 +418,13 @@ def run_extras(torch, W, B, peak, headline_job):
     out = {}
     del headline_job
     torch.cuda.empty_cache()
-    for name, steps, lp in (("resnet50_bf16", 500, True), ("resnet50_f32", 500, False), ("resnet18", 1000, False),
-                            ("vgg16", 40, False), ("tiny", 2000, False)):
-        job = BspJob(name, torch, W, B, with_lp=lp)
+    for name, steps, lp, flags in (("resnet50_bf16", 500, True, 0), ("resnet50_bf16", 500, False, B.BULK_COPY),
+                                   ("resnet50_f32", 500, False, 0), ("resnet50_f32", 500, False, B.BULK_COPY),
+                                   ("resnet18", 1000, False, 0), ("vgg16", 40, False, 0), ("tiny", 2000, False, 0)):
+        job = BspJob(name, torch, W, B, with_lp=lp, flags=flags)
         _, sched = throughput_schedule(job.cfg, 64, W, torch)
         ms, launches = job.timed(steps, 5, sched)
-        key = name + ("+lp_copy" if lp else "")
+        key = name + ("+lp_copy" if lp else "") + ("+bulk_copy_ring" if flags else "")
         out[key] = bsp_line(job, ms, steps, launches, peak)
         if name == "tiny":
             out[key]["note"] = "33.6 MB working set: L2-resident and launch-bound, not an HBM figure"

@@ -59,6 +59,10 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
 #define OMNI_UNSCALED_MEAN 1u   /* lambda_k = 1/K: the unweighted arm of the paper's "weighted aggregation" table */
 #define OMNI_ASP_NO_LR_SCALE 2u /* eta_k = eta: the "w/o LR scaling" arm of the paper's ASP table */
 #define OMNI_INPUT_IS_TIME 4u   /* measurements are compute times t_k instead of throughputs T_k */
+#define OMNI_BULK_COPY 8u       /* omni_aggregate_bsp stages its inputs through shared memory with bulk (TMA)
+                                   copies and an mbarrier ring instead of register-staged vector loads: same
+                                   results bit for bit; a bounded wait that runs out surfaces as
+                                   OMNI_ERR_TIMEOUT from omni_get_stats */
 
 /* The "Input:" line of Algorithm 1 / Algorithm 2 (K, B, Delta b_k, b_min, b_max) plus the EWMA weight. */
 typedef struct {

@@ -16,7 +16,7 @@ MAX_K = 32
 TAU_BINS = 33
 BSP, ASP = 0, 1
 F32, BF16 = 0, 1
-UNSCALED_MEAN, ASP_NO_LR_SCALE, INPUT_IS_TIME = 1, 2, 4
+UNSCALED_MEAN, ASP_NO_LR_SCALE, INPUT_IS_TIME, BULK_COPY = 1, 2, 4, 8
 
 OK = 0
 ERR_NULL, ERR_BAD_K, ERR_BAD_WORKER, ERR_BAD_BATCH, ERR_INFEASIBLE, ERR_BAD_MEASUREMENT = -1, -2, -3, -4, -5, -6

@@ -42,7 +42,7 @@ struct Workspace {
     double partials[kMaxGrid];  // one squared-norm partial per CTA
     double sqnorm;              // result cell
     unsigned int ticket;        // CTAs finished in the current launch; reset by the last one
-    unsigned int pad;
+    unsigned int status;        // set non-zero by a kernel whose bounded wait ran out
 };
 
 struct BspParams {

@@ -6,21 +6,12 @@
 #include <new>
 
 #include "controller.h"
+#include "dispatch.h"
 #include "kernels.cuh"
 
 namespace omni {
 
-using KernelFn = const void *;
-
-// A kernel instantiation with the launch geometry that goes with it.
-struct KernelInfo {
-    KernelFn fn = nullptr;
-    int threads = 0;
-    int ctas_per_sm = 0;          // wanted CTAs per SM (capped by what fits)
-    unsigned long long tile = 0;  // elements per tile
-};
-
-struct LaunchShape { int grid = 0; int block = 0; };
+struct LaunchShape { int grid = 0; int block = 0; };  // grid == 0: not yet sized for this device
 
 }  // namespace omni
 
@@ -35,6 +26,7 @@ struct omni_ctx {
     int last_cuda = 0;
     uint64_t launches = 0;
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
+    omni::LaunchShape bulk_shape[2][OMNI_MAX_K + 1];    // [dtype][K], bulk-copy ring kernel
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
     omni::LaunchShape seq_shape[2][2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][wide][M]
 };
@@ -126,7 +118,7 @@ int ensure_device(omni_ctx *ctx)
     Workspace *ws = nullptr;
     OMNI_CUDA(ctx, cudaMalloc(&ws, sizeof(Workspace)));
     cudaError_t e = cudaMemset(ws, 0, sizeof(Workspace));
-    if (e == cudaSuccess) e = cudaMallocHost(&ctx->host_cell, sizeof(double));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->host_cell, 2 * sizeof(double));
     if (e != cudaSuccess) {
         cudaFree(ws);
         ctx->last_cuda = int(e);
@@ -144,7 +136,9 @@ int shape_for(omni_ctx *ctx, const KernelInfo &ki, LaunchShape &s)
 {
     if (s.grid > 0) return OMNI_OK;
     int per_sm = 0;
-    OMNI_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ki.fn, ki.threads, 0));
+    if (ki.smem > 0)
+        OMNI_CUDA(ctx, cudaFuncSetAttribute(ki.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ki.smem)));
+    OMNI_CUDA(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ki.fn, ki.threads, ki.smem));
     if (per_sm < 1) per_sm = 1;
     if (ki.ctas_per_sm > 0 && per_sm > ki.ctas_per_sm) per_sm = ki.ctas_per_sm;
     int grid = ctx->sm_count * per_sm;
@@ -195,7 +189,7 @@ int check_buckets(const omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buc
 int launch(omni_ctx *ctx, const KernelInfo &ki, int grid, void *params, cudaStream_t stream)
 {
     void *args[] = {params};
-    OMNI_CUDA(ctx, cudaLaunchKernel(ki.fn, dim3(grid), dim3(ki.threads), args, 0, stream));
+    OMNI_CUDA(ctx, cudaLaunchKernel(ki.fn, dim3(grid), dim3(ki.threads), args, ki.smem, stream));
     ctx->launches += 1;
     return OMNI_OK;
 }
@@ -219,9 +213,10 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
                 float lr, float mu, float wd, cudaStream_t stream)
 {
     const int K = ctx->ctl.K();
+    const bool bulk = (ctx->ctl.config().flags & OMNI_BULK_COPY) != 0;
     const bool wide = all_aligned32(buckets, n_buckets, 0, K);
-    const KernelInfo ki = bsp_kernel(dtype, K, wide);
-    LaunchShape &shape = ctx->bsp_shape[dtype][wide][K];
+    const KernelInfo ki = bulk ? bulk_kernel(dtype, K) : bsp_kernel(dtype, K, wide);
+    LaunchShape &shape = bulk ? ctx->bulk_shape[dtype][K] : ctx->bsp_shape[dtype][wide][K];
     int rc = shape_for(ctx, ki, shape);
     if (rc != OMNI_OK) return rc;
     const unsigned long long tile = ki.tile;
@@ -520,9 +515,17 @@ int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream)
     if (!ctx || !out) return OMNI_ERR_NULL;
     if (ctx->ws) {
         cudaStream_t s = static_cast<cudaStream_t>(stream);
-        OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->host_cell, &ctx->ws->sqnorm, sizeof(double), cudaMemcpyDeviceToHost, s));
+        OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->host_cell, &ctx->ws->sqnorm, 2 * sizeof(double), cudaMemcpyDeviceToHost, s));
         OMNI_CUDA(ctx, cudaStreamSynchronize(s));
-        ctx->tally.grad_sqnorm = *ctx->host_cell;
+        ctx->tally.grad_sqnorm = ctx->host_cell[0];
+        unsigned int words[2];
+        std::memcpy(words, &ctx->host_cell[1], sizeof words);   // ticket, status
+        if (words[1] != 0) {
+            // a bounded device-side wait ran out in some earlier launch: report once and clear
+            OMNI_CUDA(ctx, cudaMemsetAsync(&ctx->ws->status, 0, sizeof(unsigned int), s));
+            *out = ctx->tally;
+            return OMNI_ERR_TIMEOUT;
+        }
     }
     *out = ctx->tally;
     return OMNI_OK;

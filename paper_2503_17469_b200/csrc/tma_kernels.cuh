@@ -1,0 +1,243 @@
+// Bulk-copy (TMA) variant of the synchronous fused step.
+//
+// One producer warp streams tiles of all K gradient buffers plus theta and v into a ring of
+// shared-memory stages with 1-D bulk copies (cp.async.bulk, completion counted on an mbarrier);
+// consumer warps take full stages, run the ordered FMA chain and the update out of shared
+// memory and write theta / v / the bf16 copy straight to global memory.  The amount of data in
+// flight per SM is fixed by the ring (stages x stage bytes), not by how the compiler schedules
+// loads, and every request to DRAM is a contiguous burst of 2-8 KB of one stream.
+//
+// Every wait on an mbarrier is bounded: when the limit is hit the thread records it in the
+// workspace status word and leaves the kernel; the host reports OMNI_ERR_TIMEOUT.
+// Bulk copies need 16-byte aligned addresses and sizes, which the library's alignment contract
+// gives for full tiles; the ragged last tile of a bucket is read with ordinary loads.
+#pragma once
+#include "kernels.cuh"
+
+namespace omni {
+
+constexpr unsigned kTmaWaitLimit = 1u << 22;  // try_wait attempts before giving up (seconds, far beyond any real wait)
+constexpr unsigned kStatusTimeout = 1u;
+
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long *b, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(b)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *b, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long *b)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_addr(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; false = gave up.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *b, unsigned parity)
+{
+    for (unsigned i = 0; i < kTmaWaitLimit; ++i)
+        if (mbar_try_wait(b, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, unsigned bytes, unsigned long long *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+struct TmaShape { int tile, stages, consumer_warps; };
+
+// Ring geometry per (gradient type, K).  Timing scans on B200: what matters is the size of each
+// bulk copy (4 KB or more per gradient stream is as fast as the register kernel, 2 KB costs
+// 2-3 %, 1 KB halves the bandwidth) and about 150 KB in flight per SM; more stages do not help.
+// So: the largest tile whose stage stays within 80 KB, and as many stages as make ~150 KB.
+template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
+{
+    const int per_elem = K * int(sizeof(G)) + 8;
+    int tile = 4096;
+    while (tile > 256 && tile * per_elem > 80 * 1024) tile /= 2;
+    const int stage = tile * per_elem;
+    int stages = (152 * 1024 + stage / 2) / stage;
+    if (stages < 2) stages = 2;
+    if (stages > 8) stages = 8;
+    return {tile, stages, 4};
+}
+template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int K)
+{
+    const TmaShape s = tma_shape<G>(K);
+    return unsigned(s.stages) * unsigned(s.tile) * unsigned(K * int(sizeof(G)) + 8);
+}
+
+template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE>
+__global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_constant__ BspParams p)
+{
+    constexpr int THREADS = (NCW + 1) * 32;
+    constexpr int NCT = NCW * 32;                       // consumer threads
+    constexpr int V = 16 / int(sizeof(G));              // elements per 16-byte gradient vector
+    constexpr int NV = WIDE ? 2 : 1;                    // vectors per work item (WIDE: 32-byte global stores)
+    constexpr int E = V * NV;                           // elements per work item
+    constexpr int SW = WIDE ? 8 : 4;                    // words per theta/v store
+    constexpr unsigned GB = TILE * sizeof(G);           // bytes of one gradient tile
+    constexpr unsigned FB = TILE * 4;                   // bytes of a theta or v tile
+    constexpr unsigned SB = K * GB + 2 * FB;            // bytes of one stage
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long full[STAGES], empty[STAGES];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const float lr = p.lr, mu = p.mu, wd = p.wd;
+    const bool with_v = mu != 0.0f;
+    const unsigned long long first = blockIdx.x, stride = gridDim.x;
+    const unsigned long long mine = first < p.tiles ? (p.tiles - first + stride - 1) / stride : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCW); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    double sq = 0.0;
+    if (warp == NCW) {
+        // ---------------- producer warp: lane 0 issues the copies ----------------
+        if (lane == 0) {
+            for (unsigned long long i = 0; i < mine; ++i) {
+                const int s = int(i % STAGES);
+                const unsigned long long tile = first + i * stride;
+                const int bi = find_bucket<kMaxBucketsPerLaunch>(p.bk, p.nb, tile);
+                const BucketDesc bd = p.bk[bi];
+                const unsigned long long base = (tile - bd.tile0) * TILE;
+                if (i >= STAGES && !mbar_wait(&empty[s], unsigned((i / STAGES - 1) & 1))) {
+                    atomicExch(&p.ws->status, kStatusTimeout);
+                    break;
+                }
+                if (base + TILE > bd.n) {          // ragged tile: consumers read it from global memory
+                    mbar_arrive(&full[s]);
+                    continue;
+                }
+                unsigned char *st = ring + size_t(s) * SB;
+                mbar_expect_tx(&full[s], K * GB + FB + (with_v ? FB : 0u));
+#pragma unroll
+                for (int k = 0; k < K; ++k) bulk_load(st + k * GB, static_cast<const G *>(p.g[bi][k]) + base, GB, &full[s]);
+                bulk_load(st + K * GB, bd.theta + base, FB, &full[s]);
+                if (with_v) bulk_load(st + K * GB + FB, bd.v + base, FB, &full[s]);
+            }
+        }
+    } else {
+        // ---------------- consumer warps ----------------
+        for (unsigned long long i = 0; i < mine; ++i) {
+            const int s = int(i % STAGES);
+            const unsigned long long tile = first + i * stride;
+            const int bi = find_bucket<kMaxBucketsPerLaunch>(p.bk, p.nb, tile);
+            const BucketDesc bd = p.bk[bi];
+            const unsigned long long base = (tile - bd.tile0) * TILE;
+            const bool has_v = bd.v != nullptr, has_lp = bd.lp != nullptr;
+            if (!mbar_wait(&full[s], unsigned((i / STAGES) & 1))) {
+                atomicExch(&p.ws->status, kStatusTimeout);
+                break;
+            }
+            if (base + TILE <= bd.n) {
+                const unsigned char *st = ring + size_t(s) * SB;
+                const float *sth = reinterpret_cast<const float *>(st + K * GB);
+                const float *sv = reinterpret_cast<const float *>(st + K * GB + FB);
+#pragma unroll 1
+                for (int j = tid; j < TILE / E; j += NCT) {
+                    float acc[E], th[E], vv[E];
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[e] = 0.0f;
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        const float lam = p.lam[k];
+#pragma unroll
+                        for (int h = 0; h < NV; ++h) {
+                            const uint4 r = *reinterpret_cast<const uint4 *>(st + k * GB + size_t(j * NV + h) * 16);
+                            Raw<4> raw; raw.w[0] = r.x; raw.w[1] = r.y; raw.w[2] = r.z; raw.w[3] = r.w;
+                            float gk[V];
+                            widen<G, 4>(raw, gk);
+#pragma unroll
+                            for (int e = 0; e < V; ++e) acc[h * V + e] = __fmaf_rn(lam, gk[e], acc[h * V + e]);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < E / 4; ++q) {
+                        const float4 t4 = *reinterpret_cast<const float4 *>(sth + j * E + 4 * q);
+                        th[4 * q] = t4.x; th[4 * q + 1] = t4.y; th[4 * q + 2] = t4.z; th[4 * q + 3] = t4.w;
+                        if (with_v) {
+                            const float4 v4 = *reinterpret_cast<const float4 *>(sv + j * E + 4 * q);
+                            vv[4 * q] = v4.x; vv[4 * q + 1] = v4.y; vv[4 * q + 2] = v4.z; vv[4 * q + 3] = v4.w;
+                        }
+                    }
+                    float part[NV];
+#pragma unroll
+                    for (int h = 0; h < NV; ++h) {
+                        part[h] = 0.0f;
+#pragma unroll
+                        for (int e = 0; e < V; ++e) {
+                            part[h] = __fmaf_rn(acc[h * V + e], acc[h * V + e], part[h]);
+                            th[h * V + e] = update_one(acc[h * V + e], th[h * V + e], vv[h * V + e], lr, mu, wd);
+                        }
+                        sq += (double)part[h];
+                    }
+                    const unsigned long long off = base + (unsigned long long)j * E;
+                    store_floats<SW, E / SW>(bd.theta + off, th);
+                    if (has_v) store_floats<SW, E / SW>(bd.v + off, vv);
+                    if (has_lp) store_lp<E / 2>(bd.lp + off, th);
+                }
+            } else {
+                // ragged tile from global memory: whole 16-byte vectors, then single elements
+                for (unsigned long long off = base + (unsigned long long)tid * V; off < bd.n; off += (unsigned long long)NCT * V) {
+                    if (off + V <= bd.n) {
+                        float acc[V], th[V], vv[V];
+#pragma unroll
+                        for (int e = 0; e < V; ++e) acc[e] = 0.0f;
+#pragma unroll
+                        for (int k = 0; k < K; ++k) {
+                            const Raw<4> raw = ld_ro<4>(static_cast<const G *>(p.g[bi][k]) + off);
+                            float gk[V];
+                            widen<G, 4>(raw, gk);
+                            const float lam = p.lam[k];
+#pragma unroll
+                            for (int e = 0; e < V; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
+                        }
+                        load_floats<4, V / 4>(bd.theta + off, th);
+                        if (with_v) load_floats<4, V / 4>(bd.v + off, vv);
+                        float part = 0.0f;
+#pragma unroll
+                        for (int e = 0; e < V; ++e) {
+                            part = __fmaf_rn(acc[e], acc[e], part);
+                            th[e] = update_one(acc[e], th[e], vv[e], lr, mu, wd);
+                        }
+                        sq += (double)part;
+                        store_floats<4, V / 4>(bd.theta + off, th);
+                        if (has_v) store_floats<4, V / 4>(bd.v + off, vv);
+                        if (has_lp) store_lp<V / 2>(bd.lp + off, th);
+                    } else {
+                        for (unsigned long long j = off; j < bd.n; ++j) {
+                            float acc = 0.0f;
+#pragma unroll
+                            for (int k = 0; k < K; ++k)
+                                acc = __fmaf_rn(p.lam[k], widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
+                            float vj = with_v ? __ldcs(bd.v + j) : 0.0f;
+                            const float t = update_one(acc, __ldcs(bd.theta + j), vj, lr, mu, wd);
+                            sq += (double)(acc * acc);
+                            bd.theta[j] = t;
+                            if (has_v) bd.v[j] = vj;
+                            if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                        }
+                    }
+                }
+            }
+            // this warp is done with the stage
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[s]);
+        }
+    }
+    finish_sqnorm<THREADS>(sq, p.ws, p.accumulate);
+}
+
+}  // namespace omni
