@@ -115,7 +115,7 @@ def measured_peak():
 
 def kernel_source_hash() -> str:
     h = hashlib.sha256()
-    for f in ("kernels.cuh", "omni.cu"):
+    for f in ("kernels.cuh", "tma_kernels.cuh", "bulk_dispatch.cu", "omni.cu"):
         h.update((ROOT / "paper_2503_17469_b200" / "csrc" / f).read_bytes())
     return h.hexdigest()[:16]
 
@@ -400,8 +400,8 @@ def main():
             "pct_of_nominal_8TBs": 100 * line_main["frac_of_nominal_8TBs"],
             "roofline": {"bound": "hbm", "achieved": line_main["achieved_gbs"], "peak": peak, "unit": "GB/s",
                          "frac": line_main["frac_of_measured"], "peak_source": f"of {peak_kind}",
-                         "kernel": "bsp_fused_kernel<bf16,16>", "bytes_per_launch": job.bytes_per_step,
-                         "traffic": recorded_traffic("bsp_fused_bf16_k16")},
+                         "kernel": "bsp_tma_kernel<bf16,16,tile 2048,2 stages>" if block == 160 else "bsp_fused_kernel<bf16,16>", "bytes_per_launch": job.bytes_per_step,
+                         "traffic": recorded_traffic("bsp_tma_bf16_k16" if block == 160 else "bsp_fused_bf16_k16")},
             "e2e": {"value": world * cfg.P * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": 8, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": launches,
@@ -418,13 +418,14 @@ def run_extras(torch, W, B, peak, headline_job):
     out = {}
     del headline_job
     torch.cuda.empty_cache()
-    for name, steps, lp, flags in (("resnet50_bf16", 500, True, 0), ("resnet50_bf16", 500, False, B.BULK_COPY),
-                                   ("resnet50_f32", 500, False, 0), ("resnet50_f32", 500, False, B.BULK_COPY),
+    for name, steps, lp, flags in (("resnet50_bf16", 500, True, 0),
+                                   ("resnet50_bf16", 500, False, B.NO_BULK_COPY),
+                                   ("resnet50_f32", 500, False, 0), ("resnet50_f32", 500, False, B.NO_BULK_COPY),
                                    ("resnet18", 1000, False, 0), ("vgg16", 40, False, 0), ("tiny", 2000, False, 0)):
         job = BspJob(name, torch, W, B, with_lp=lp, flags=flags)
         _, sched = throughput_schedule(job.cfg, 64, W, torch)
         ms, launches = job.timed(steps, 5, sched)
-        key = name + ("+lp_copy" if lp else "") + ("+bulk_copy_ring" if flags else "")
+        key = name + ("+lp_copy" if lp else "") + ("+register_kernels" if flags else "")
         out[key] = bsp_line(job, ms, steps, launches, peak)
         if name == "tiny":
             out[key]["note"] = "33.6 MB working set: L2-resident and launch-bound, not an HBM figure"

@@ -16,7 +16,8 @@ MAX_K = 32
 TAU_BINS = 33
 BSP, ASP = 0, 1
 F32, BF16 = 0, 1
-UNSCALED_MEAN, ASP_NO_LR_SCALE, INPUT_IS_TIME, BULK_COPY = 1, 2, 4, 8
+UNSCALED_MEAN, ASP_NO_LR_SCALE, INPUT_IS_TIME, BULK_COPY, NO_BULK_COPY = 1, 2, 4, 8, 16
+DEFAULT_FLAGS = 0  # OR-ed into every new context's flags (the tests use it to force a kernel family)
 
 OK = 0
 ERR_NULL, ERR_BAD_K, ERR_BAD_WORKER, ERR_BAD_BATCH, ERR_INFEASIBLE, ERR_BAD_MEASUREMENT = -1, -2, -3, -4, -5, -6
@@ -187,7 +188,7 @@ class Omni:
         self._h = C.c_void_p()
         self.K = K
         self.global_batch = global_batch
-        cfg = omni_config(K, global_batch, b_min, b_max, deadband, ewma_alpha, mode, flags)
+        cfg = omni_config(K, global_batch, b_min, b_max, deadband, ewma_alpha, mode, flags | DEFAULT_FLAGS)
         self._check(lib().omni_create(C.byref(cfg), C.byref(self._h)))
         self._i32K = C.c_int32 * K
         self._f64K = C.c_double * K

@@ -25,8 +25,33 @@ template <typename G> KernelInfo bulk_for(int K)
     return {};
 }
 
+template <typename G, int M> KernelInfo bulk_seq_info()
+{
+    constexpr TmaShape sh = tma_shape<G>(M);
+    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, M, sh.tile, sh.stages, sh.consumer_warps, false, true>),
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(M)};
+}
+
+template <typename G> KernelInfo bulk_seq_for(int M)
+{
+    switch (M) {
+#define OMNI_CASE(k) case k: return bulk_seq_info<G, k>();
+        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
+        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
+#undef OMNI_CASE
+    }
+    return {};
+}
+
 }  // namespace
 
 KernelInfo bulk_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bulk_for<__nv_bfloat16>(K) : bulk_for<float>(K); }
+KernelInfo bulk_seq_kernel(int dtype, int M) { return dtype == OMNI_BF16 ? bulk_seq_for<__nv_bfloat16>(M) : bulk_seq_for<float>(M); }
+
+bool bulk_preferred(int dtype, int streams)
+{
+    const TmaShape sh = dtype == OMNI_BF16 ? tma_shape<__nv_bfloat16>(streams) : tma_shape<float>(streams);
+    return sh.tile * (dtype == OMNI_BF16 ? 2 : 4) >= 4096;
+}
 
 }  // namespace omni

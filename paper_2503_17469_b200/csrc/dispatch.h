@@ -14,7 +14,12 @@ struct KernelInfo {
     unsigned smem = 0;            // dynamic shared memory per CTA, bytes
 };
 
-// Bulk-copy ring variant of the synchronous step (bulk_dispatch.cu).
+// Bulk-copy ring kernels (bulk_dispatch.cu): the synchronous step for K workers, and the
+// asynchronous apply of M queued arrivals (M = 1: a single arrival; M <= OMNI_MAX_ASP_BATCH).
 KernelInfo bulk_kernel(int dtype, int K);
+KernelInfo bulk_seq_kernel(int dtype, int M);
+// Whether the ring is the better choice for this many streams: its bulk copies must be at least
+// 4 KB each to match the register-staged kernels (smaller copies lose DRAM efficiency).
+bool bulk_preferred(int dtype, int streams);
 
 }  // namespace omni

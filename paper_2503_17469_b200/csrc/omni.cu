@@ -27,6 +27,7 @@ struct omni_ctx {
     uint64_t launches = 0;
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
     omni::LaunchShape bulk_shape[2][OMNI_MAX_K + 1];    // [dtype][K], bulk-copy ring kernel
+    omni::LaunchShape bulk_seq_shape[2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][M]
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
     omni::LaunchShape seq_shape[2][2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][wide][M]
 };
@@ -148,6 +149,27 @@ int shape_for(omni_ctx *ctx, const KernelInfo &ki, LaunchShape &s)
     return OMNI_OK;
 }
 
+// Kernel family for a call with this many gradient streams: the flags force one, otherwise the
+// bulk-copy ring runs wherever its copies are large enough.
+bool use_bulk(const omni_ctx *ctx, int dtype, int streams)
+{
+    const uint32_t f = ctx->ctl.config().flags;
+    if (f & OMNI_NO_BULK_COPY) return false;
+    if (f & OMNI_BULK_COPY) return true;
+    return bulk_preferred(dtype, streams);
+}
+
+// Asynchronous applies: timing on B200 puts the single arrival (and two arrivals with momentum)
+// on the register-staged kernels and larger batches on the ring.
+bool use_bulk_seq(const omni_ctx *ctx, int dtype, int m, bool momentum)
+{
+    const uint32_t f = ctx->ctl.config().flags;
+    if (f & OMNI_NO_BULK_COPY) return false;
+    if (f & OMNI_BULK_COPY) return true;
+    if (m < 2 || (m == 2 && momentum)) return false;
+    return bulk_preferred(dtype, m);
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
@@ -213,7 +235,7 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
                 float lr, float mu, float wd, cudaStream_t stream)
 {
     const int K = ctx->ctl.K();
-    const bool bulk = (ctx->ctl.config().flags & OMNI_BULK_COPY) != 0;
+    const bool bulk = use_bulk(ctx, dtype, K);
     const bool wide = all_aligned32(buckets, n_buckets, 0, K);
     const KernelInfo ki = bulk ? bulk_kernel(dtype, K) : bsp_kernel(dtype, K, wide);
     LaunchShape &shape = bulk ? ctx->bulk_shape[dtype][K] : ctx->bsp_shape[dtype][wide][K];
@@ -341,6 +363,51 @@ static int check_bsp_batches(const omni_ctx *ctx, const int32_t *b)
     return OMNI_OK;
 }
 
+// m queued arrivals applied in one pass (m = 1: a single arrival), bulk-copy ring or registers.
+static int enqueue_seq(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t dtype, int32_t m,
+                       const int32_t *workers, const int32_t *b_used, float lr, float momentum, float weight_decay,
+                       cudaStream_t stream)
+{
+    const bool bulk = use_bulk_seq(ctx, dtype, m, momentum != 0.0f);
+    bool wide = true;
+    for (int i = 0; i < m; ++i) wide = wide && all_aligned32(buckets, n_buckets, workers[i], workers[i] + 1);
+    const KernelInfo ki = bulk ? bulk_seq_kernel(dtype, m) : seq_kernel(dtype, m, wide);
+    LaunchShape &shape = bulk ? ctx->bulk_seq_shape[dtype][m] : ctx->seq_shape[dtype][wide][m];
+    int rc = shape_for(ctx, ki, shape);
+    if (rc != OMNI_OK) return rc;
+
+    BspParams p;
+    int i = 0;
+    while (i < n_buckets) {
+        std::memset(&p, 0, sizeof p);
+        unsigned long long tiles = 0;
+        int nb = 0;
+        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+            const omni_bucket &bk = buckets[i];
+            if (bk.n == 0) continue;
+            p.bk[nb] = {static_cast<float *>(bk.param), static_cast<float *>(bk.momentum),
+                        static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
+            for (int a = 0; a < m; ++a) p.g[nb][a] = bk.grads[workers[a]];
+            tiles += (bk.n + ki.tile - 1) / ki.tile;
+            ++nb;
+        }
+        if (nb == 0) break;
+        // Eq. 5b per arrival: eta = lr * b_used / B, in double, rounded once to float
+        for (int a = 0; a < m; ++a)
+            p.lam[a] = float((ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
+                                 ? double(lr)
+                                 : double(lr) * double(b_used[a]) / double(ctx->ctl.B()));
+        p.mu = momentum; p.wd = weight_decay;
+        p.nb = nb;
+        p.tiles = tiles;
+        p.ws = ctx->ws;
+        const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
+        rc = launch(ctx, ki, grid, &p, stream);
+        if (rc != OMNI_OK) return rc;
+    }
+    return OMNI_OK;
+}
+
 int omni_aggregate_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                        const int32_t *b, float lr, float momentum, float weight_decay, void *stream)
 {
@@ -412,6 +479,16 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
     const double eta_k = (ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
                              ? double(lr)
                              : double(lr) * double(b_used) / double(ctx->ctl.B());
+    if (use_bulk_seq(ctx, grad_dtype, 1, momentum != 0.0f)) {
+        // the ring kernel in sequential mode with one arrival
+        rc = enqueue_seq(ctx, buckets, n_buckets, grad_dtype, 1, &worker, &b_used, lr, momentum, weight_decay,
+                         static_cast<cudaStream_t>(stream));
+        if (rc != OMNI_OK) return rc;
+        ctx->tally.arrivals += 1;
+        ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
+        if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+        return OMNI_OK;
+    }
     const bool wide = all_aligned32(buckets, n_buckets, worker, worker + 1);
     const KernelInfo ki = asp_kernel(grad_dtype, wide, momentum != 0.0f);
     LaunchShape &shape = ctx->asp_shape[grad_dtype][wide][momentum != 0.0f];
@@ -466,42 +543,9 @@ int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_bu
     rc = ensure_device(ctx);
     if (rc != OMNI_OK) return rc;
 
-    bool wide = true;
-    for (int i = 0; i < m; ++i) wide = wide && all_aligned32(buckets, n_buckets, workers[i], workers[i] + 1);
-    const KernelInfo ki = seq_kernel(grad_dtype, m, wide);
-    LaunchShape &shape = ctx->seq_shape[grad_dtype][wide][m];
-    rc = shape_for(ctx, ki, shape);
+    rc = enqueue_seq(ctx, buckets, n_buckets, grad_dtype, m, workers, b_used, lr, momentum, weight_decay,
+                     static_cast<cudaStream_t>(stream));
     if (rc != OMNI_OK) return rc;
-
-    BspParams p;
-    int i = 0;
-    while (i < n_buckets) {
-        std::memset(&p, 0, sizeof p);
-        unsigned long long tiles = 0;
-        int nb = 0;
-        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
-            const omni_bucket &bk = buckets[i];
-            if (bk.n == 0) continue;
-            p.bk[nb] = {static_cast<float *>(bk.param), static_cast<float *>(bk.momentum),
-                        static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
-            for (int a = 0; a < m; ++a) p.g[nb][a] = bk.grads[workers[a]];
-            tiles += (bk.n + ki.tile - 1) / ki.tile;
-            ++nb;
-        }
-        if (nb == 0) break;
-        // Eq. 5b per arrival: eta = lr * b_used / B, in double, rounded once to float
-        for (int a = 0; a < m; ++a)
-            p.lam[a] = float((ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
-                                 ? double(lr)
-                                 : double(lr) * double(b_used[a]) / double(ctx->ctl.B()));
-        p.mu = momentum; p.wd = weight_decay;
-        p.nb = nb;
-        p.tiles = tiles;
-        p.ws = ctx->ws;
-        const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
-        rc = launch(ctx, ki, grid, &p, static_cast<cudaStream_t>(stream));
-        if (rc != OMNI_OK) return rc;
-    }
     for (int a = 0; a < m; ++a) {
         ctx->tally.arrivals += 1;
         ctx->tally.tau_hist[tau[a] < OMNI_TAU_BINS - 1 ? tau[a] : OMNI_TAU_BINS - 1] += 1;
@@ -540,8 +584,9 @@ int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *gri
     if (grad_dtype != OMNI_F32 && grad_dtype != OMNI_BF16) return OMNI_ERR_BAD_CONFIG;
     int rc = ensure_device(ctx);
     if (rc != OMNI_OK) return rc;
-    LaunchShape &shape = ctx->bsp_shape[grad_dtype][1][K];
-    rc = shape_for(ctx, bsp_kernel(grad_dtype, K, true), shape);
+    const bool bulk = use_bulk(ctx, grad_dtype, K);
+    LaunchShape &shape = bulk ? ctx->bulk_shape[grad_dtype][K] : ctx->bsp_shape[grad_dtype][1][K];
+    rc = shape_for(ctx, bulk ? bulk_kernel(grad_dtype, K) : bsp_kernel(grad_dtype, K, true), shape);
     if (rc != OMNI_OK) return rc;
     *grid = shape.grid;
     *block = shape.block;

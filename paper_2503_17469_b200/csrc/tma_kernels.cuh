@@ -7,6 +7,10 @@
 // flight per SM is fixed by the ring (stages x stage bytes), not by how the compiler schedules
 // loads, and every request to DRAM is a contiguous burst of 2-8 KB of one stream.
 //
+// SEQ = true is the asynchronous apply on the same ring: the K streams are K queued arrivals
+// (K = 1: a single arrival), lam[k] carries eta_k, and each element goes through the K
+// per-arrival updates in order instead of one weighted sum and one update; no norm is produced.
+//
 // Every wait on an mbarrier is bounded: when the limit is hit the thread records it in the
 // workspace status word and leaves the kernel; the host reports OMNI_ERR_TIMEOUT.
 // Bulk copies need 16-byte aligned addresses and sizes, which the library's alignment contract
@@ -75,7 +79,7 @@ template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int 
     return unsigned(s.stages) * unsigned(s.tile) * unsigned(K * int(sizeof(G)) + 8);
 }
 
-template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE>
+template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false>
 __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_constant__ BspParams p)
 {
     constexpr int THREADS = (NCW + 1) * 32;
@@ -147,22 +151,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                 const float *sv = reinterpret_cast<const float *>(st + K * GB + FB);
 #pragma unroll 1
                 for (int j = tid; j < TILE / E; j += NCT) {
-                    float acc[E], th[E], vv[E];
-#pragma unroll
-                    for (int e = 0; e < E; ++e) acc[e] = 0.0f;
-#pragma unroll
-                    for (int k = 0; k < K; ++k) {
-                        const float lam = p.lam[k];
-#pragma unroll
-                        for (int h = 0; h < NV; ++h) {
-                            const uint4 r = *reinterpret_cast<const uint4 *>(st + k * GB + size_t(j * NV + h) * 16);
-                            Raw<4> raw; raw.w[0] = r.x; raw.w[1] = r.y; raw.w[2] = r.z; raw.w[3] = r.w;
-                            float gk[V];
-                            widen<G, 4>(raw, gk);
-#pragma unroll
-                            for (int e = 0; e < V; ++e) acc[h * V + e] = __fmaf_rn(lam, gk[e], acc[h * V + e]);
-                        }
-                    }
+                    float th[E], vv[E];
 #pragma unroll
                     for (int q = 0; q < E / 4; ++q) {
                         const float4 t4 = *reinterpret_cast<const float4 *>(sth + j * E + 4 * q);
@@ -172,16 +161,48 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                             vv[4 * q] = v4.x; vv[4 * q + 1] = v4.y; vv[4 * q + 2] = v4.z; vv[4 * q + 3] = v4.w;
                         }
                     }
-                    float part[NV];
+                    if constexpr (SEQ) {
 #pragma unroll
-                    for (int h = 0; h < NV; ++h) {
-                        part[h] = 0.0f;
+                        for (int k = 0; k < K; ++k) {
+                            const float eta = p.lam[k];
 #pragma unroll
-                        for (int e = 0; e < V; ++e) {
-                            part[h] = __fmaf_rn(acc[h * V + e], acc[h * V + e], part[h]);
-                            th[h * V + e] = update_one(acc[h * V + e], th[h * V + e], vv[h * V + e], lr, mu, wd);
+                            for (int h = 0; h < NV; ++h) {
+                                const uint4 r = *reinterpret_cast<const uint4 *>(st + k * GB + size_t(j * NV + h) * 16);
+                                Raw<4> raw; raw.w[0] = r.x; raw.w[1] = r.y; raw.w[2] = r.z; raw.w[3] = r.w;
+                                float gk[V];
+                                widen<G, 4>(raw, gk);
+#pragma unroll
+                                for (int e = 0; e < V; ++e)
+                                    th[h * V + e] = update_one(gk[e], th[h * V + e], vv[h * V + e], eta, mu, wd);
+                            }
                         }
-                        sq += (double)part[h];
+                    } else {
+                        float acc[E];
+#pragma unroll
+                        for (int e = 0; e < E; ++e) acc[e] = 0.0f;
+#pragma unroll
+                        for (int k = 0; k < K; ++k) {
+                            const float lam = p.lam[k];
+#pragma unroll
+                            for (int h = 0; h < NV; ++h) {
+                                const uint4 r = *reinterpret_cast<const uint4 *>(st + k * GB + size_t(j * NV + h) * 16);
+                                Raw<4> raw; raw.w[0] = r.x; raw.w[1] = r.y; raw.w[2] = r.z; raw.w[3] = r.w;
+                                float gk[V];
+                                widen<G, 4>(raw, gk);
+#pragma unroll
+                                for (int e = 0; e < V; ++e) acc[h * V + e] = __fmaf_rn(lam, gk[e], acc[h * V + e]);
+                            }
+                        }
+#pragma unroll
+                        for (int h = 0; h < NV; ++h) {
+                            float part = 0.0f;
+#pragma unroll
+                            for (int e = 0; e < V; ++e) {
+                                part = __fmaf_rn(acc[h * V + e], acc[h * V + e], part);
+                                th[h * V + e] = update_one(acc[h * V + e], th[h * V + e], vv[h * V + e], lr, mu, wd);
+                            }
+                            sq += (double)part;
+                        }
                     }
                     const unsigned long long off = base + (unsigned long long)j * E;
                     store_floats<SW, E / SW>(bd.theta + off, th);
@@ -192,39 +213,59 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                 // ragged tile from global memory: whole 16-byte vectors, then single elements
                 for (unsigned long long off = base + (unsigned long long)tid * V; off < bd.n; off += (unsigned long long)NCT * V) {
                     if (off + V <= bd.n) {
-                        float acc[V], th[V], vv[V];
+                        float th[V], vv[V];
+                        Raw<4> raw[K];
 #pragma unroll
-                        for (int e = 0; e < V; ++e) acc[e] = 0.0f;
-#pragma unroll
-                        for (int k = 0; k < K; ++k) {
-                            const Raw<4> raw = ld_ro<4>(static_cast<const G *>(p.g[bi][k]) + off);
-                            float gk[V];
-                            widen<G, 4>(raw, gk);
-                            const float lam = p.lam[k];
-#pragma unroll
-                            for (int e = 0; e < V; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
-                        }
+                        for (int k = 0; k < K; ++k) raw[k] = ld_ro<4>(static_cast<const G *>(p.g[bi][k]) + off);
                         load_floats<4, V / 4>(bd.theta + off, th);
                         if (with_v) load_floats<4, V / 4>(bd.v + off, vv);
-                        float part = 0.0f;
+                        if constexpr (SEQ) {
 #pragma unroll
-                        for (int e = 0; e < V; ++e) {
-                            part = __fmaf_rn(acc[e], acc[e], part);
-                            th[e] = update_one(acc[e], th[e], vv[e], lr, mu, wd);
+                            for (int k = 0; k < K; ++k) {
+                                float gk[V];
+                                widen<G, 4>(raw[k], gk);
+#pragma unroll
+                                for (int e = 0; e < V; ++e) th[e] = update_one(gk[e], th[e], vv[e], p.lam[k], mu, wd);
+                            }
+                        } else {
+                            float acc[V];
+#pragma unroll
+                            for (int e = 0; e < V; ++e) acc[e] = 0.0f;
+#pragma unroll
+                            for (int k = 0; k < K; ++k) {
+                                float gk[V];
+                                widen<G, 4>(raw[k], gk);
+                                const float lam = p.lam[k];
+#pragma unroll
+                                for (int e = 0; e < V; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
+                            }
+                            float part = 0.0f;
+#pragma unroll
+                            for (int e = 0; e < V; ++e) {
+                                part = __fmaf_rn(acc[e], acc[e], part);
+                                th[e] = update_one(acc[e], th[e], vv[e], lr, mu, wd);
+                            }
+                            sq += (double)part;
                         }
-                        sq += (double)part;
                         store_floats<4, V / 4>(bd.theta + off, th);
                         if (has_v) store_floats<4, V / 4>(bd.v + off, vv);
                         if (has_lp) store_lp<V / 2>(bd.lp + off, th);
                     } else {
                         for (unsigned long long j = off; j < bd.n; ++j) {
-                            float acc = 0.0f;
-#pragma unroll
-                            for (int k = 0; k < K; ++k)
-                                acc = __fmaf_rn(p.lam[k], widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
                             float vj = with_v ? __ldcs(bd.v + j) : 0.0f;
-                            const float t = update_one(acc, __ldcs(bd.theta + j), vj, lr, mu, wd);
-                            sq += (double)(acc * acc);
+                            float t = __ldcs(bd.theta + j);
+                            if constexpr (SEQ) {
+#pragma unroll
+                                for (int k = 0; k < K; ++k)
+                                    t = update_one(widen1<G>(static_cast<const G *>(p.g[bi][k]), j), t, vj, p.lam[k], mu, wd);
+                            } else {
+                                float acc = 0.0f;
+#pragma unroll
+                                for (int k = 0; k < K; ++k)
+                                    acc = __fmaf_rn(p.lam[k], widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
+                                t = update_one(acc, t, vj, lr, mu, wd);
+                                sq += (double)(acc * acc);
+                            }
                             bd.theta[j] = t;
                             if (has_v) bd.v[j] = vj;
                             if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
@@ -237,7 +278,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
             if (lane == 0) mbar_arrive(&empty[s]);
         }
     }
-    finish_sqnorm<THREADS>(sq, p.ws, p.accumulate);
+    if constexpr (!SEQ) finish_sqnorm<THREADS>(sq, p.ws, p.accumulate);
 }
 
 }  // namespace omni
