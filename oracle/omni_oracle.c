@@ -421,6 +421,36 @@ void oracle_asp_apply_f32(uint64_t n, const void *g, int dtype_bf16, int32_t b_u
     }
 }
 
+/* Algorithm 2 taken literally: the worker pulled the server parameters some updates ago (its
+ * snapshot), computes theta_k = snapshot - eta_k g on its replica and pushes theta_k, and the
+ * server OVERWRITES its parameters with it, so whatever other workers pushed since the pull is
+ * lost.  theta (out) never enters the arithmetic.  Plain SGD as in Algorithm 2; the optional
+ * weight-decay term acts on the replica: d = g + wd * snapshot. */
+void oracle_asp_push_overwrite_f64(uint64_t n, const void *g, int dtype_bf16, int32_t b_used, int32_t B,
+                                   uint32_t flags, double *theta, const double *snapshot, double lr, double wd)
+{
+    double eta_k = oracle_asp_lr(lr, b_used, B, flags);
+    const void *gp[1] = { g };
+    for (uint64_t j = 0; j < n; ++j) {
+        double d = grad_at(gp, dtype_bf16, 0, j) + wd * snapshot[j];
+        theta[j] = snapshot[j] - eta_k * d;
+    }
+}
+
+void oracle_asp_push_overwrite_f32(uint64_t n, const void *g, int dtype_bf16, int32_t b_used, int32_t B,
+                                   uint32_t flags, float *theta, const float *snapshot, uint16_t *theta_lp,
+                                   float lr, float wd)
+{
+    float eta_k = (float)oracle_asp_lr((double)lr, b_used, B, flags);
+    const void *gp[1] = { g };
+    for (uint64_t j = 0; j < n; ++j) {
+        float gj = (float)grad_at(gp, dtype_bf16, 0, j);
+        float d = wd != 0.0f ? fmaf(wd, snapshot[j], gj) : gj;
+        theta[j] = fmaf(-eta_k, d, snapshot[j]);
+        if (theta_lp) theta_lp[j] = float_to_bf16(theta[j]);
+    }
+}
+
 /* Staleness bookkeeping of the arrival stream: tau = server updates since the worker's last
  * read.  The paper defines no staleness-dependent factor, so tau is tallied, never multiplied in.
  * hist has 33 bins: 0..31 and one overflow bin. */

@@ -70,6 +70,10 @@ def lib() -> C.CDLL:
         L.oracle_asp_apply_f64.restype = None
         L.oracle_asp_apply_f32.argtypes = [u64, vp, C.c_int, i32, i32, u32, vp, vp, vp, f32, f32, f32]
         L.oracle_asp_apply_f32.restype = None
+        L.oracle_asp_push_overwrite_f64.argtypes = [u64, vp, C.c_int, i32, i32, u32, vp, vp, f64, f64]
+        L.oracle_asp_push_overwrite_f64.restype = None
+        L.oracle_asp_push_overwrite_f32.argtypes = [u64, vp, C.c_int, i32, i32, u32, vp, vp, vp, f32, f32]
+        L.oracle_asp_push_overwrite_f32.restype = None
         L.oracle_tau_record.argtypes = [vp, vp, i32]
         L.oracle_tau_record.restype = None
         _lib = L
@@ -222,6 +226,23 @@ def asp_apply_f32(g, b_used, B, theta, v, lr, mu, wd, flags=0, theta_lp=None) ->
     assert v is not None or mu == 0
     lib().oracle_asp_apply_f32(g.shape[0], _ptr(g), int(g.dtype == np.uint16), b_used, B, flags,
                                _ptr(theta), _ptr(v), _ptr(theta_lp), lr, mu, wd)
+
+
+def asp_push_overwrite_f64(g, b_used, B, theta, snapshot, lr, wd=0.0, flags=0) -> None:
+    """Algorithm 2 literally: theta (server, overwritten) <- snapshot - eta_k * g."""
+    assert g.dtype in (np.float32, np.uint16) and g.flags.c_contiguous
+    _chk(theta, np.float64), _chk(snapshot, np.float64)
+    assert theta.shape == snapshot.shape == g.shape
+    lib().oracle_asp_push_overwrite_f64(g.shape[0], _ptr(g), int(g.dtype == np.uint16), b_used, B, flags,
+                                        _ptr(theta), _ptr(snapshot), lr, wd)
+
+
+def asp_push_overwrite_f32(g, b_used, B, theta, snapshot, lr, wd=0.0, flags=0, theta_lp=None) -> None:
+    assert g.dtype in (np.float32, np.uint16) and g.flags.c_contiguous
+    _chk(theta, np.float32), _chk(snapshot, np.float32)
+    assert theta.shape == snapshot.shape == g.shape
+    lib().oracle_asp_push_overwrite_f32(g.shape[0], _ptr(g), int(g.dtype == np.uint16), b_used, B, flags,
+                                        _ptr(theta), _ptr(snapshot), _ptr(theta_lp), lr, wd)
 
 
 class TauStats:

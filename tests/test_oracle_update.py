@@ -252,3 +252,43 @@ def test_staleness_is_tallied_not_applied():
         s.record(tau)
     assert s.hist[0] == 2 and s.hist[5] == 1 and s.hist[31] == 1 and s.hist[32] == 2
     assert s.hist.sum() == 6 and s.tau_max == 100
+
+
+def test_overwrite_semantics_hand_case():
+    """Algorithm 2 literally: a push replaces the server copy by snapshot - eta_k g, so what
+    arrived since the worker's pull is lost; applying the same gradients instead keeps both."""
+    c = GOLD["asp_overwrite"]
+    for dt, push, apply_ in ((np.float32, O.asp_push_overwrite_f32, O.asp_apply_f32),
+                             (np.float64, O.asp_push_overwrite_f64, O.asp_apply_f64)):
+        theta = _f(c["theta0"], dt)
+        applied = _f(c["theta0"], dt)
+        for ev in c["events"]:
+            push(_f(ev["g"], np.float32), ev["b_used"], c["B"], theta, _f(ev["snapshot"], dt), c["lr"])
+            assert theta.tolist() == ev["theta_after"]
+            apply_(_f(ev["g"], np.float32), ev["b_used"], c["B"], applied, None, c["lr"], 0.0, 0.0)
+        assert applied.tolist() == c["apply_semantics_would_give"]
+
+
+def test_overwrite_equals_apply_when_nothing_arrived_in_between():
+    rng = np.random.default_rng(91)
+    n = 2001
+    g = rng.normal(0, 1e-3, n).astype(np.float32)
+    for dt, push, apply_ in ((np.float32, O.asp_push_overwrite_f32, O.asp_apply_f32),
+                             (np.float64, O.asp_push_overwrite_f64, O.asp_apply_f64)):
+        server = rng.normal(0, 0.05, n).astype(dt)
+        a, b = server.copy(), server.copy()
+        push(g, 24, 512, a, server.copy(), 0.1, 1e-3)
+        apply_(g, 24, 512, b, None, 0.1, 0.0, 1e-3)
+        assert np.array_equal(a, b)
+
+
+def test_overwrite_ignores_the_current_server_copy():
+    rng = np.random.default_rng(92)
+    n = 500
+    g = rng.normal(0, 1e-3, n).astype(np.float32)
+    snap = rng.normal(0, 0.05, n)
+    out1, out2 = rng.normal(0, 1, n), np.zeros(n)
+    O.asp_push_overwrite_f64(g, 16, 128, out1, snap, 0.1)
+    O.asp_push_overwrite_f64(g, 16, 128, out2, snap, 0.1)
+    assert np.array_equal(out1, out2)
+    np.testing.assert_allclose(out1, snap - 0.1 * 16 / 128 * g.astype(np.float64), rtol=1e-14, atol=1e-18)
