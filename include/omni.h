@@ -173,6 +173,24 @@ int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_bu
                          const int32_t *workers, const int32_t *b_used, const int32_t *tau, float lr, float momentum,
                          float weight_decay, void *stream);
 
+/* Algorithm 2 taken literally (pull / local update / push with overwrite), for callers that want
+ * the paper's parameter-server semantics instead of "apply to the current copy".
+ * omni_asp_pull: pullFromPS -- snapshots[i] (HOST array of n_buckets device pointers, float[n]
+ * each, 16-byte aligned, caller-owned, one set per worker) <- buckets[i].param, by device copies
+ * enqueued on `stream`.
+ * omni_asp_push_overwrite: the worker's local step and pushToPS in one launch --
+ *   theta_j <- fma(-eta_k, d, s_j),  d = weight_decay ? fma(weight_decay, s_j, g_j) : g_j,
+ * with s the snapshot that worker pulled, g = buckets[i].grads[worker], eta_k as in omni_apply_asp.
+ * The server copy is OVERWRITTEN: whatever other workers pushed since this worker's pull is lost
+ * (the paper's "overridden" updates), so here the staleness tau changes the result, although it
+ * still enters no formula; it is tallied as in omni_apply_asp.  Plain SGD as in Algorithm 2 (no
+ * momentum buffer is read or written).  With tau = 0 the result equals omni_apply_asp's.
+ * Errors: NULL, BAD_WORKER, BAD_BATCH, BAD_TAU, ALIGN, BAD_CONFIG, CUDA. */
+int omni_asp_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, void *const *snapshots, void *stream);
+int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                            int32_t worker, int32_t b_used, int32_t tau, const void *const *snapshots, float lr,
+                            float weight_decay, void *stream);
+
 /* Same step as omni_aggregate_bsp for gradients that arrive in HOST memory (pinned memory gives
  * asynchronous copies).  host_grads: host array of n_buckets*K host pointers, entry [i*K + k] =
  * worker k's gradient for bucket i.  buckets[i].grads must point at K device staging buffers of

@@ -27,7 +27,7 @@ EXPORTS = (
     "omni_strerror", "omni_create", "omni_destroy", "omni_get_batches", "omni_set_batches",
     "omni_rebatch", "omni_asp_report", "omni_rebatch_static", "omni_aggregate_bsp",
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
-    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch",
+    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
     L.omni_apply_asp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, f32, f32, f32, vp]
     L.omni_apply_asp_batch.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, C.POINTER(i32), C.POINTER(i32),
                                        C.POINTER(i32), f32, f32, f32, vp]
+    L.omni_asp_pull.argtypes = [vp, C.POINTER(omni_bucket), i32, C.POINTER(vp), vp]
+    L.omni_asp_push_overwrite.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, C.POINTER(vp), f32, f32, vp]
     L.omni_aggregate_bsp_host.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(vp), C.POINTER(i32),
                                           f32, f32, f32, vp, C.POINTER(C.c_double)]
     L.omni_get_stats.argtypes = [vp, C.POINTER(omni_stats), vp]
@@ -274,6 +276,25 @@ class Omni:
         self._check(lib().omni_apply_asp_batch(self._h, buckets.array, buckets.n_buckets, buckets.dtype, m,
                                                arr(*workers), arr(*b_used), arr(*tau), lr, momentum, weight_decay,
                                                self._stream(stream)))
+
+    @staticmethod
+    def _ptr_table(tensors):
+        tab = (C.c_void_p * max(1, len(tensors)))()
+        for i, t in enumerate(tensors):
+            tab[i] = t.data_ptr()
+        return tab
+
+    def asp_pull(self, buckets: BucketSet, snapshots: Sequence, stream=None) -> None:
+        """pullFromPS: ``snapshots[i]`` (float32 CUDA tensor per bucket) <- the server parameters."""
+        self._check(lib().omni_asp_pull(self._h, buckets.array, buckets.n_buckets, self._ptr_table(snapshots),
+                                        self._stream(stream)))
+
+    def asp_push_overwrite(self, buckets: BucketSet, worker: int, b_used: int, tau: int, snapshots: Sequence,
+                           lr: float, weight_decay: float = 0.0, stream=None) -> None:
+        """Algorithm 2 literally: server parameters <- snapshot - eta_k * gradient (overwrite)."""
+        self._check(lib().omni_asp_push_overwrite(self._h, buckets.array, buckets.n_buckets, buckets.dtype, worker,
+                                                  b_used, tau, self._ptr_table(snapshots), lr, weight_decay,
+                                                  self._stream(stream)))
 
     def stats(self, stream=None) -> Stats:
         s = omni_stats()

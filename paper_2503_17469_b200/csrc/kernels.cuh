@@ -517,4 +517,69 @@ __global__ void __launch_bounds__(THREADS) asp_batch_kernel(const __grid_constan
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Asynchronous push with overwrite (Algorithm 2 taken literally): the server copy is replaced by
+// snapshot - eta_k * (g + wd * snapshot), where snapshot is what the worker pulled earlier.
+// Reads snapshot and g, writes theta (and the bf16 copy): 12 bytes per parameter.
+// ---------------------------------------------------------------------------------------------
+struct OverwriteParams {
+    BucketDesc bk[kMaxBucketsPerLaunch];      // theta = destination; v unused
+    const void *g[kMaxBucketsPerLaunch];
+    const float *snap[kMaxBucketsPerLaunch];
+    float eta, wd;
+    int nb;
+    unsigned long long tiles;
+};
+
+template <typename G, int THREADS, int C, bool WIDE>
+__global__ void __launch_bounds__(THREADS) asp_overwrite_kernel(const __grid_constant__ OverwriteParams p)
+{
+    using Ge = Geo<G, WIDE>;
+    constexpr int E = Ge::E;
+    constexpr unsigned long long TILE = (unsigned long long)THREADS * E * C;
+    const int tid = threadIdx.x;
+    const float eta = p.eta, wd = p.wd;
+
+    for (unsigned long long tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
+        const int bi = find_bucket<kMaxBucketsPerLaunch>(p.bk, p.nb, tile);
+        const BucketDesc bd = p.bk[bi];
+        const G *g = static_cast<const G *>(p.g[bi]);
+        const float *snap = p.snap[bi];
+        const unsigned long long base = (tile - bd.tile0) * TILE;
+        const bool has_lp = bd.lp != nullptr;
+
+        if (base + TILE <= bd.n) {
+            Raw<Ge::GW> raw[C];
+            float th[C][E];
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                raw[c] = ld_ro<Ge::GW>(g + off);
+                load_floats<Ge::FW, Ge::FN>(snap + off, th[c]);
+            }
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                float gk[E], unused;
+                widen<G, Ge::GW>(raw[c], gk);
+#pragma unroll
+                for (int e = 0; e < E; ++e) th[c][e] = update_one(gk[e], th[c][e], unused, eta, 0.0f, wd);
+                store_floats<Ge::FW, Ge::FN>(bd.theta + off, th[c]);
+                if (has_lp) store_lp<Ge::LW>(bd.lp + off, th[c]);
+            }
+        } else {
+#pragma unroll 1
+            for (int c = 0; c < C; ++c) {
+                const unsigned long long off = base + (unsigned long long)(c * THREADS + tid) * E;
+                for (unsigned long long j = off; j < bd.n && j < off + E; ++j) {
+                    float unused;
+                    const float t = update_one(widen1<G>(g, j), __ldcs(snap + j), unused, eta, 0.0f, wd);
+                    bd.theta[j] = t;
+                    if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                }
+            }
+        }
+    }
+}
+
 }  // namespace omni

@@ -29,6 +29,7 @@ struct omni_ctx {
     omni::LaunchShape bulk_shape[2][OMNI_MAX_K + 1];    // [dtype][K], bulk-copy ring kernel
     omni::LaunchShape bulk_seq_shape[2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][M]
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
+    omni::LaunchShape overwrite_shape[2][2];            // [dtype][wide]
     omni::LaunchShape seq_shape[2][2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][wide][M]
 };
 
@@ -91,6 +92,17 @@ KernelInfo seq_kernel(int dtype, int M, bool wide)
 {
     if (dtype == OMNI_BF16) return wide ? seq_kernel_for<__nv_bfloat16, true>(M) : seq_kernel_for<__nv_bfloat16, false>(M);
     return wide ? seq_kernel_for<float, true>(M) : seq_kernel_for<float, false>(M);
+}
+
+template <typename G, bool WIDE> KernelInfo overwrite_info()
+{
+    return {reinterpret_cast<KernelFn>(&asp_overwrite_kernel<G, kAspThreads, kAspChunks, WIDE>), kAspThreads,
+            asp_ctas_per_sm(false), (unsigned long long)kAspThreads * Geo<G, WIDE>::E * kAspChunks};
+}
+KernelInfo overwrite_kernel(int dtype, bool wide)
+{
+    if (dtype == OMNI_BF16) return wide ? overwrite_info<__nv_bfloat16, true>() : overwrite_info<__nv_bfloat16, false>();
+    return wide ? overwrite_info<float, true>() : overwrite_info<float, false>();
 }
 
 template <typename G, bool WIDE> KernelInfo asp_info(bool momentum)
@@ -551,6 +563,80 @@ int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_bu
         ctx->tally.tau_hist[tau[a] < OMNI_TAU_BINS - 1 ? tau[a] : OMNI_TAU_BINS - 1] += 1;
         if (tau[a] > ctx->tally.tau_max) ctx->tally.tau_max = tau[a];
     }
+    return OMNI_OK;
+}
+
+int omni_asp_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, void *const *snapshots, void *stream)
+{
+    if (!ctx || (n_buckets > 0 && (!buckets || !snapshots))) return OMNI_ERR_NULL;
+    if (n_buckets < 0) return OMNI_ERR_BAD_CONFIG;
+    for (int i = 0; i < n_buckets; ++i) {
+        if (buckets[i].n == 0) continue;
+        if (!buckets[i].param || !snapshots[i]) return OMNI_ERR_NULL;
+        if (!aligned16(buckets[i].param) || !aligned16(snapshots[i])) return OMNI_ERR_ALIGN;
+    }
+    for (int i = 0; i < n_buckets; ++i)
+        if (buckets[i].n)
+            OMNI_CUDA(ctx, cudaMemcpyAsync(snapshots[i], buckets[i].param, buckets[i].n * sizeof(float),
+                                           cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+    return OMNI_OK;
+}
+
+int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                            int32_t worker, int32_t b_used, int32_t tau, const void *const *snapshots, float lr,
+                            float weight_decay, void *stream)
+{
+    if (!ctx) return OMNI_ERR_NULL;
+    const int K = ctx->ctl.K();
+    if (worker < 0 || worker >= K) return OMNI_ERR_BAD_WORKER;
+    if (b_used < 1) return OMNI_ERR_BAD_BATCH;
+    if (tau < 0) return OMNI_ERR_BAD_TAU;
+    if (n_buckets > 0 && !snapshots) return OMNI_ERR_NULL;
+    int rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, worker, 0.0f);
+    if (rc != OMNI_OK) return rc;
+    bool wide = all_aligned32(buckets, n_buckets, worker, worker + 1);
+    for (int i = 0; i < n_buckets; ++i) {
+        if (buckets[i].n == 0) continue;
+        if (!snapshots[i]) return OMNI_ERR_NULL;
+        if (!aligned16(snapshots[i])) return OMNI_ERR_ALIGN;
+        wide = wide && aligned32(snapshots[i]);
+    }
+    rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    const double eta_k = (ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
+                             ? double(lr)
+                             : double(lr) * double(b_used) / double(ctx->ctl.B());
+    const KernelInfo ki = overwrite_kernel(grad_dtype, wide);
+    LaunchShape &shape = ctx->overwrite_shape[grad_dtype][wide];
+    rc = shape_for(ctx, ki, shape);
+    if (rc != OMNI_OK) return rc;
+
+    OverwriteParams p;
+    int i = 0;
+    while (i < n_buckets) {
+        std::memset(&p, 0, sizeof p);
+        unsigned long long tiles = 0;
+        int nb = 0;
+        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+            const omni_bucket &bk = buckets[i];
+            if (bk.n == 0) continue;
+            p.bk[nb] = {static_cast<float *>(bk.param), nullptr, static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
+            p.g[nb] = bk.grads[worker];
+            p.snap[nb] = static_cast<const float *>(snapshots[i]);
+            tiles += (bk.n + ki.tile - 1) / ki.tile;
+            ++nb;
+        }
+        if (nb == 0) break;
+        p.eta = float(eta_k); p.wd = weight_decay;
+        p.nb = nb;
+        p.tiles = tiles;
+        const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
+        rc = launch(ctx, ki, grid, &p, static_cast<cudaStream_t>(stream));
+        if (rc != OMNI_OK) return rc;
+    }
+    ctx->tally.arrivals += 1;
+    ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
+    if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
     return OMNI_OK;
 }
 

@@ -322,6 +322,61 @@ def test_asp_batched_apply_equals_successive_arrivals(kind, mu, wd):
     assert L.omni_apply_asp_batch(h, bs.array, 1, bs.dtype, 2, i32(0, 1), i32(8, 8), i32(0, -1), 0.1, mu, wd, None) == B.ERR_BAD_TAU
 
 
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+def test_asp_pull_and_push_with_overwrite(kind):
+    """Algorithm 2 literally on a shrunk model: workers pull snapshots at different times and
+    push with overwrite; the event stream (with controller feedback) runs on both sides; the
+    server copy matches the oracle bit for bit after every event, and differs from what applying
+    the same gradients would give."""
+    base = W.config("resnet50_asp")
+    cfg = W.scaled(W.Config(**{**base.__dict__, "grad_dtype": kind}), 500)
+    buf = W.make_buffers(cfg, DEV)
+    lay = buf.layout
+    K = cfg.K
+    o = B.Omni(K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, 1.0, B.ASP)
+    ora = O.Controller(K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, 1.0, O.MODE_ASP)
+    lp = torch.zeros(lay.total, dtype=torch.bfloat16, device=DEV)
+    bs = B.BucketSet.from_flat(lay, buf.theta, buf.grads, None, lp)
+    sl = [slice(bk.start, bk.start + bk.n) for bk in lay.buckets]
+    snaps = [torch.zeros(lay.total, device=DEV) for _ in range(K)]           # one snapshot set per worker
+    th_o = to_np(buf.theta)
+    lp_o = np.zeros(lay.total, np.uint16)
+    snaps_o = [np.zeros(lay.total, np.float32) for _ in range(K)]
+    applied = th_o.copy()
+    g_np = [to_np(g) for g in buf.grads]
+    for k in range(K):                                                        # everybody pulls theta_0
+        o.asp_pull(bs, [snaps[k][s] for s in sl])
+        snaps_o[k][:] = th_o
+    gen = torch.Generator().manual_seed(cfg.seed)
+    T = W.draw_throughputs(K, gen, cfg.ratio)
+    u = torch.rand(300, generator=gen, dtype=torch.float64).tolist()
+    b = [cfg.global_batch // K] * K
+    last = [0] * K
+    tally = O.TauStats()
+    for i in range(300):
+        k = W.pick_worker(u[i], [T[j] / b[j] for j in range(K)])
+        tau = i - last[k]
+        o.asp_push_overwrite(bs, k, b[k], tau, [snaps[k][s] for s in sl], cfg.lr, 1e-4)
+        o.asp_pull(bs, [snaps[k][s] for s in sl])                             # next iteration starts with a pull
+        for s in sl:                                                          # the oracle walks the same buckets
+            O.asp_push_overwrite_f32(g_np[k][s], b[k], cfg.global_batch, th_o[s], snaps_o[k][s], cfg.lr, 1e-4, theta_lp=lp_o[s])
+        snaps_o[k][:] = th_o
+        O.asp_apply_f32(g_np[k], b[k], cfg.global_batch, applied, None, cfg.lr, 0.0, 1e-4)
+        tally.record(tau)
+        last[k] = i + 1
+        nb = o.asp_report(k, b[k], T[k])
+        assert nb == ora.asp_report(k, b[k], T[k])
+        b[k] = nb
+        if i % 50 == 0 or i == 299:
+            assert np.array_equal(to_np(buf.theta), th_o), i
+    assert np.array_equal(to_np(lp), lp_o)
+    assert np.array_equal(to_np(snaps[3]), snaps_o[3])
+    st = o.stats()
+    assert st.arrivals == 300 and st.tau_hist == tally.hist.tolist() and st.tau_max == tally.tau_max
+    real = np.concatenate([np.arange(a, a + n) for _, a, n in lay.tensor_slices()])
+    assert np.abs(th_o[real] - applied[real]).max() > 1e-5      # overwriting loses updates that applying keeps
+
+
 def test_asp_no_lr_scale_flag():
     n = 10_000
     theta, _, grads, _ = _make(2, n, "f32", 8, momentum=False)
