@@ -240,6 +240,14 @@ int omni_aggregate_bsp_noalloc(int32_t K, const omni_bucket *buckets, int32_t n_
 /* Synchronises `stream` and fills *out (host). */
 int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream);
 
+/* Failure-path self-test (no counterpart in the paper).  Every device-side wait of the library is
+ * bounded; when one runs out the kernel records it and the next omni_get_stats returns
+ * OMNI_ERR_TIMEOUT once, then clears the record.  This call enqueues a one-warp kernel that waits,
+ * with a short limit, on a barrier nothing completes, so that the path can be observed without
+ * any kernel misbehaving: afterwards omni_get_stats must return OMNI_ERR_TIMEOUT, the context
+ * stays usable, and the following omni_get_stats returns OMNI_OK.  Errors: NULL, CUDA. */
+int omni_selftest_wait_expiry(omni_ctx *ctx, void *stream);
+
 /* The cudaError_t of the last failed CUDA call made through this context (0 if none). */
 int omni_last_cuda_error(const omni_ctx *ctx);
 

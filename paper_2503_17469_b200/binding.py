@@ -27,7 +27,7 @@ EXPORTS = (
     "omni_strerror", "omni_create", "omni_destroy", "omni_get_batches", "omni_set_batches",
     "omni_rebatch", "omni_asp_report", "omni_rebatch_static", "omni_aggregate_bsp",
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
-    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite",
+    "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
     L.omni_aggregate_bsp_host.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(vp), C.POINTER(i32),
                                           f32, f32, f32, vp, C.POINTER(C.c_double)]
     L.omni_get_stats.argtypes = [vp, C.POINTER(omni_stats), vp]
+    L.omni_selftest_wait_expiry.argtypes = [vp, vp]
     L.omni_last_cuda_error.argtypes = [vp]
     L.omni_query_launch.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
     L.omni_kernel_launches.argtypes = [vp]
@@ -301,6 +302,10 @@ class Omni:
         st = C.c_void_p(0) if stream is None and not self._device_used() else self._stream(stream)
         self._check(lib().omni_get_stats(self._h, C.byref(s), st))
         return Stats(s.grad_sqnorm, s.weight_sum, s.steps, s.arrivals, list(s.tau_hist), s.tau_max)
+
+    def selftest_wait_expiry(self, stream=None) -> None:
+        """Enqueue the diagnostic kernel whose bounded wait runs out (next ``stats()`` raises TIMEOUT)."""
+        self._check(lib().omni_selftest_wait_expiry(self._h, self._stream(stream)))
 
     def _device_used(self) -> bool:
         return lib().omni_kernel_launches(self._h) > 0

@@ -48,6 +48,12 @@ template <typename G> KernelInfo bulk_seq_for(int M)
 KernelInfo bulk_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bulk_for<__nv_bfloat16>(K) : bulk_for<float>(K); }
 KernelInfo bulk_seq_kernel(int dtype, int M) { return dtype == OMNI_BF16 ? bulk_seq_for<__nv_bfloat16>(M) : bulk_seq_for<float>(M); }
 
+int launch_expire_wait(void *workspace, unsigned attempts, void *stream)
+{
+    expire_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<Workspace *>(workspace), attempts);
+    return int(cudaGetLastError());
+}
+
 bool bulk_preferred(int dtype, int streams)
 {
     const TmaShape sh = dtype == OMNI_BF16 ? tma_shape<__nv_bfloat16>(streams) : tma_shape<float>(streams);

@@ -22,4 +22,7 @@ KernelInfo bulk_seq_kernel(int dtype, int M);
 // 4 KB each to match the register-staged kernels (smaller copies lose DRAM efficiency).
 bool bulk_preferred(int dtype, int streams);
 
+// Launches the bounded-wait diagnostic kernel (bulk_dispatch.cu); returns the cudaError_t as int.
+int launch_expire_wait(void *workspace, unsigned attempts, void *stream);
+
 }  // namespace omni

@@ -661,6 +661,20 @@ int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream)
     return OMNI_OK;
 }
 
+int omni_selftest_wait_expiry(omni_ctx *ctx, void *stream)
+{
+    if (!ctx) return OMNI_ERR_NULL;
+    int rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    const int e = launch_expire_wait(ctx->ws, 2048u, stream);
+    if (e != 0) {
+        ctx->last_cuda = e;
+        return OMNI_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return OMNI_OK;
+}
+
 int omni_last_cuda_error(const omni_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
 
 int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *grid, int32_t *block)

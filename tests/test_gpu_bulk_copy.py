@@ -95,3 +95,26 @@ def test_bulk_copy_headline_config_full_size():
     st = o.stats()
     assert abs(st.grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
     assert np.array_equal(to_np(buf.theta), th_o) and np.array_equal(to_np(buf.v), v_o)
+
+
+def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
+    """A wait that runs out sets the status word; omni_get_stats reports OMNI_ERR_TIMEOUT once,
+    clears it, and the context keeps working (no trap, no hang, no lost context)."""
+    K, n = 4, 30_000
+    theta, v, grads, _ = _make(K, n, "bf16", 5)
+    o = B.Omni(K, 64, 1, 64, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    b = [16] * K
+    o.aggregate_bsp(bs, b, 0.1, 0.9)
+    assert o.stats().steps == 1
+    o.selftest_wait_expiry()
+    with pytest.raises(B.OmniError) as e:
+        o.stats()
+    assert e.value.status == B.ERR_TIMEOUT
+    st = o.stats()                       # reported once, then cleared
+    assert st.steps == 1
+    th_o, v_o, g_np = to_np(theta.t), to_np(v.t), [to_np(g.t) for g in grads]
+    o.aggregate_bsp(bs, b, 0.1, 0.9)     # still usable, still correct
+    sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 0.0)
+    assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+    assert np.array_equal(to_np(theta.t), th_o)
