@@ -44,7 +44,9 @@ _lib = None
 def lib() -> C.CDLL:
     global _lib
     if _lib is None:
-        L = C.CDLL(str(build()))
+        # OMNI_ORACLE_LIB: load this build of the oracle instead (used by the test that plants
+        # mistakes in copies of the source to show that the pins catch them)
+        L = C.CDLL(os.environ.get("OMNI_ORACLE_LIB") or str(build()))
         vp, i32, u32, u64, f64, f32 = C.c_void_p, C.c_int32, C.c_uint32, C.c_uint64, C.c_double, C.c_float
         L.oracle_ctl_sizeof.restype = C.c_size_t
         L.oracle_ctl_init.argtypes = [vp, i32, i32, i32, i32, f64, f64, i32, u32]
