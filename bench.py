@@ -320,6 +320,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="omni", choices=["omni", "reference"])
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--extras", default="all", choices=["all", "none", "asp"],
+                    help="which of the other configurations to time as well (not part of `value`)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -379,8 +381,8 @@ def main():
     del host
 
     extras = {}
-    if rank == 0 and world == 1 and not args.no_extras:
-        extras = run_extras(torch, W, B, peak, job)
+    if rank == 0 and world == 1 and not args.no_extras and args.extras != "none":
+        extras = run_extras(torch, W, B, peak, job, only_asp=args.extras == "asp")
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -413,7 +415,7 @@ def main():
     ranks.close()
 
 
-def run_extras(torch, W, B, peak, headline_job):
+def run_extras(torch, W, B, peak, headline_job, only_asp=False):
     """The other configurations, each timed with CUDA events after warm-up (not part of `value`)."""
     out = {}
     del headline_job
@@ -422,6 +424,8 @@ def run_extras(torch, W, B, peak, headline_job):
                                    ("resnet50_bf16", 500, False, B.NO_BULK_COPY),
                                    ("resnet50_f32", 500, False, 0), ("resnet50_f32", 500, False, B.NO_BULK_COPY),
                                    ("resnet18", 1000, False, 0), ("vgg16", 40, False, 0), ("tiny", 2000, False, 0)):
+        if only_asp:
+            break
         job = BspJob(name, torch, W, B, with_lp=lp, flags=flags)
         _, sched = throughput_schedule(job.cfg, 64, W, torch)
         ms, launches = job.timed(steps, 5, sched)
