@@ -433,6 +433,29 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
         out[key] = bsp_line(job, ms, steps, launches, peak)
         if name == "tiny":
             out[key]["note"] = "33.6 MB working set: L2-resident and launch-bound, not an HBM figure"
+            # the same steps with the launches captured once in a CUDA graph (fixed batches)
+            b = job.omni.batches
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                job.omni.aggregate_bsp(job.buckets, b, job.cfg.lr, job.cfg.momentum)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(50):
+                    job.omni.aggregate_bsp(job.buckets, b, job.cfg.lr, job.cfg.momentum)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(40):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            gms = e0.elapsed_time(e1)
+            out[key + "+cuda_graph"] = bsp_line(job, gms, 2000, 2000, peak)
+            out[key + "+cuda_graph"]["note"] = "50 steps per graph, fixed batches; L2-resident"
+            del graph
         del job
         torch.cuda.empty_cache()
     # asynchronous arrivals: 1000 single-worker gradients with controller feedback

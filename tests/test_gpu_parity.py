@@ -234,6 +234,34 @@ def test_results_are_deterministic():
     assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
 
 
+def test_steps_replayed_from_a_cuda_graph():
+    """Ten steps captured once into a CUDA graph (after one eager call, which binds the context
+    to the device and sizes its launches) and replayed twice: the same bits as thirty eager
+    steps of the oracle, and the norm of the last step."""
+    K, n = 4, 1 << 18
+    theta, v, grads, _ = _make(K, n, "f32", 321)
+    o = B.Omni(K, 64, 2, 48, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    b = [2, 6, 19, 37]
+    th_o, v_o, g_np = to_np(theta.t), to_np(v.t), [to_np(g.t) for g in grads]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(10):                      # eager warm-up on the capture stream
+            o.aggregate_bsp(bs, b, 0.1, 0.9)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for _ in range(10):
+            o.aggregate_bsp(bs, b, 0.1, 0.9)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    for _ in range(30):
+        sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 0.0)
+    assert np.array_equal(to_np(theta.t), th_o) and np.array_equal(to_np(v.t), v_o)
+    assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+
+
 def test_host_gradient_entry_point():
     K, n = 4, 70_001
     theta, v, grads, _ = _make(K, n, "bf16", 11)
