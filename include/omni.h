@@ -60,9 +60,9 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
 #define OMNI_ASP_NO_LR_SCALE 2u /* eta_k = eta: the "w/o LR scaling" arm of the paper's ASP table */
 #define OMNI_INPUT_IS_TIME 4u   /* measurements are compute times t_k instead of throughputs T_k */
 /* Kernel family.  By default the device calls stage their inputs through shared memory with
- * bulk (TMA) copies and an mbarrier ring wherever each copy is at least 4 KB (up to about 20
- * gradient streams), and use register-staged 128/256-bit loads otherwise; a single asynchronous
- * arrival always takes the register-staged kernel, which measured faster.  The two flags force
+ * bulk (TMA) copies and an mbarrier ring (the synchronous step for every K, asynchronous batches
+ * of three or more arrivals); a single asynchronous arrival, and two arrivals with momentum, take
+ * the register-staged 128/256-bit-load kernels, which measured faster there.  The two flags force
  * one family; results are the same bit for bit.  A bounded wait of the ring that runs out
  * surfaces as OMNI_ERR_TIMEOUT from omni_get_stats. */
 #define OMNI_BULK_COPY 8u
@@ -252,8 +252,8 @@ int omni_selftest_wait_expiry(omni_ctx *ctx, void *stream);
 int omni_last_cuda_error(const omni_ctx *ctx);
 
 /* Persistent-grid size and block size the synchronous kernel for this K and dtype is launched
- * with on the current device (32-byte aligned buffers assumed; block = 160 means the bulk-copy
- * ring: 4 consumer warps + 1 producer warp), and the number of kernels enqueued so far. */
+ * with on the current device (32-byte aligned buffers assumed; block = 288 means the bulk-copy
+ * ring: 8 consumer warps + 1 producer warp), and the number of kernels enqueued so far. */
 int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *grid, int32_t *block);
 uint64_t omni_kernel_launches(const omni_ctx *ctx);
 

@@ -57,7 +57,7 @@ int launch_expire_wait(void *workspace, unsigned attempts, void *stream)
 bool bulk_preferred(int dtype, int streams)
 {
     const TmaShape sh = dtype == OMNI_BF16 ? tma_shape<__nv_bfloat16>(streams) : tma_shape<float>(streams);
-    return sh.tile * (dtype == OMNI_BF16 ? 2 : 4) >= 4096;
+    return sh.tile * (dtype == OMNI_BF16 ? 2 : 4) >= 2048;
 }
 
 }  // namespace omni

@@ -19,7 +19,8 @@ struct KernelInfo {
 KernelInfo bulk_kernel(int dtype, int K);
 KernelInfo bulk_seq_kernel(int dtype, int M);
 // Whether the ring is the better choice for this many streams: its bulk copies must be at least
-// 4 KB each to match the register-staged kernels (smaller copies lose DRAM efficiency).
+// 2 KB each (true for every K up to OMNI_MAX_K with the current ring geometry; 1 KB copies halve
+// the bandwidth).
 bool bulk_preferred(int dtype, int streams);
 
 // Launches the bounded-wait diagnostic kernel (bulk_dispatch.cu); returns the cudaError_t as int.

@@ -61,7 +61,9 @@ struct TmaShape { int tile, stages, consumer_warps; };
 // Ring geometry per (gradient type, K).  Timing scans on B200: what matters is the size of each
 // bulk copy (4 KB or more per gradient stream is as fast as the register kernel, 2 KB costs
 // 2-3 %, 1 KB halves the bandwidth) and about 150 KB in flight per SM; more stages do not help.
-// So: the largest tile whose stage stays within 80 KB, and as many stages as make ~150 KB.
+// So: the largest tile whose stage stays within 80 KB, and as many stages as make ~150 KB
+// (halving the stage size or a 110 KB ring cost 3-5 % in back-to-back runs).  Eight consumer
+// warps: 4 were 1-3 % slower, 6-12 the same, 16 slower again on bf16.
 template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
 {
     const int per_elem = K * int(sizeof(G)) + 8;
@@ -71,7 +73,7 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
     int stages = (152 * 1024 + stage / 2) / stage;
     if (stages < 2) stages = 2;
     if (stages > 8) stages = 8;
-    return {tile, stages, 4};
+    return {tile, stages, 8};
 }
 template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int K)
 {
