@@ -60,9 +60,11 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
 #define OMNI_ASP_NO_LR_SCALE 2u /* eta_k = eta: the "w/o LR scaling" arm of the paper's ASP table */
 #define OMNI_INPUT_IS_TIME 4u   /* measurements are compute times t_k instead of throughputs T_k */
 /* Kernel family.  By default the device calls stage their inputs through shared memory with
- * bulk (TMA) copies and an mbarrier ring (the synchronous step for every K, asynchronous batches
- * of three or more arrivals); a single asynchronous arrival, and two arrivals with momentum, take
- * the register-staged 128/256-bit-load kernels, which measured faster there.  The two flags force
+ * bulk (TMA) copies and an mbarrier ring; register-staged 128/256-bit-load kernels exist for
+ * every call as well (and serve omni_aggregate_bsp_noalloc and omni_asp_push_overwrite).  The ring
+ * kernels also alternate the direction in which successive calls walk the parameters and keep
+ * theta and v in L2 with evict-last priority, so that a call finds the part its predecessor
+ * touched last still in cache.  The two flags force
  * one family; results are the same bit for bit.  A bounded wait of the ring that runs out
  * surfaces as OMNI_ERR_TIMEOUT from omni_get_stats. */
 #define OMNI_BULK_COPY 8u

@@ -52,6 +52,7 @@ struct BspParams {
     float lr, mu, wd;
     int nb;
     int accumulate;  // 0: sqnorm = sum of this launch; 1: sqnorm += sum (later launch of one call)
+    int reverse;     // walk the tiles from the last to the first (see omni.cu: alternating sweeps)
     unsigned long long tiles;
     Workspace *ws;
 };

@@ -25,6 +25,7 @@ struct omni_ctx {
     int sm_count = 0;
     int last_cuda = 0;
     uint64_t launches = 0;
+    unsigned sweep = 0;              // calls that walked the parameters so far (parity = sweep direction)
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
     omni::LaunchShape bulk_shape[2][OMNI_MAX_K + 1];    // [dtype][K], bulk-copy ring kernel
     omni::LaunchShape bulk_seq_shape[2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][M]
@@ -171,16 +172,8 @@ bool use_bulk(const omni_ctx *ctx, int dtype, int streams)
     return bulk_preferred(dtype, streams);
 }
 
-// Asynchronous applies: timing on B200 puts the single arrival (and two arrivals with momentum)
-// on the register-staged kernels and larger batches on the ring.
-bool use_bulk_seq(const omni_ctx *ctx, int dtype, int m, bool momentum)
-{
-    const uint32_t f = ctx->ctl.config().flags;
-    if (f & OMNI_NO_BULK_COPY) return false;
-    if (f & OMNI_BULK_COPY) return true;
-    if (m < 2 || (m == 2 && momentum)) return false;
-    return bulk_preferred(dtype, m);
-}
+// Asynchronous applies take the same decision with the number of queued arrivals as stream count.
+bool use_bulk_seq(const omni_ctx *ctx, int dtype, int m, bool /*momentum*/) { return use_bulk(ctx, dtype, m); }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
@@ -275,6 +268,7 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
         p.lr = lr; p.mu = mu; p.wd = wd;
         p.nb = nb;
         p.accumulate = launched > 0;
+        p.reverse = int(ctx->sweep & 1u);
         p.tiles = tiles;
         p.ws = ctx->ws;
         const unsigned long long want = tiles < 1 ? 1 : tiles;
@@ -283,6 +277,10 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
         if (rc != OMNI_OK) return rc;
         ++launched;
     }
+    // Alternate the sweep direction from call to call: the parameters and momentum touched last
+    // are the ones still in L2 (loaded and stored with evict-last priority), so the next call
+    // starts where this one ended and finds part of them there instead of in DRAM.
+    ctx->sweep += 1;
     return OMNI_OK;
 }
 
@@ -411,12 +409,14 @@ static int enqueue_seq(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buck
                                  : double(lr) * double(b_used[a]) / double(ctx->ctl.B()));
         p.mu = momentum; p.wd = weight_decay;
         p.nb = nb;
+        p.reverse = int(ctx->sweep & 1u);
         p.tiles = tiles;
         p.ws = ctx->ws;
         const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
         rc = launch(ctx, ki, grid, &p, stream);
         if (rc != OMNI_OK) return rc;
     }
+    ctx->sweep += 1;
     return OMNI_OK;
 }
 

@@ -50,10 +50,34 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *b, unsigned parity
         if (mbar_try_wait(b, parity)) return true;
     return false;
 }
-__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, unsigned bytes, unsigned long long *bar)
+// L2 eviction policies: gradients are read once (evict first); theta and v come back in the
+// next launch (evict last), see the alternating sweeps in omni.cu.
+__device__ __forceinline__ unsigned long long policy_evict_first()
 {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ unsigned long long policy_evict_last()
+{
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, unsigned bytes, unsigned long long *bar,
+                                          unsigned long long policy)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy) : "memory");
+}
+// 16-byte stores of floats with an L2 policy
+template <int N> __device__ __forceinline__ void store_floats_policy(float *p, const float *o, unsigned long long policy)
+{
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i)
+        asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1,%2,%3,%4}, %5;"
+                     ::"l"(p + 4 * i), "r"(__float_as_uint(o[4 * i])), "r"(__float_as_uint(o[4 * i + 1])),
+                       "r"(__float_as_uint(o[4 * i + 2])), "r"(__float_as_uint(o[4 * i + 3])), "l"(policy) : "memory");
 }
 
 struct TmaShape { int tile, stages, consumer_warps; };
@@ -100,6 +124,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
     const float lr = p.lr, mu = p.mu, wd = p.wd;
     const bool with_v = mu != 0.0f;
     const unsigned long long first = blockIdx.x, stride = gridDim.x;
+    const unsigned long long pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
     const unsigned long long mine = first < p.tiles ? (p.tiles - first + stride - 1) / stride : 0;
 
     if (tid == 0) {
@@ -114,7 +139,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
         if (lane == 0) {
             for (unsigned long long i = 0; i < mine; ++i) {
                 const int s = int(i % STAGES);
-                const unsigned long long tile = first + i * stride;
+                const unsigned long long t = first + i * stride;
+                const unsigned long long tile = p.reverse ? p.tiles - 1 - t : t;
                 const int bi = find_bucket<kMaxBucketsPerLaunch>(p.bk, p.nb, tile);
                 const BucketDesc bd = p.bk[bi];
                 const unsigned long long base = (tile - bd.tile0) * TILE;
@@ -129,16 +155,17 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                 unsigned char *st = ring + size_t(s) * SB;
                 mbar_expect_tx(&full[s], K * GB + FB + (with_v ? FB : 0u));
 #pragma unroll
-                for (int k = 0; k < K; ++k) bulk_load(st + k * GB, static_cast<const G *>(p.g[bi][k]) + base, GB, &full[s]);
-                bulk_load(st + K * GB, bd.theta + base, FB, &full[s]);
-                if (with_v) bulk_load(st + K * GB + FB, bd.v + base, FB, &full[s]);
+                for (int k = 0; k < K; ++k) bulk_load(st + k * GB, static_cast<const G *>(p.g[bi][k]) + base, GB, &full[s], pol_stream);
+                bulk_load(st + K * GB, bd.theta + base, FB, &full[s], pol_keep);
+                if (with_v) bulk_load(st + K * GB + FB, bd.v + base, FB, &full[s], pol_keep);
             }
         }
     } else {
         // ---------------- consumer warps ----------------
         for (unsigned long long i = 0; i < mine; ++i) {
             const int s = int(i % STAGES);
-            const unsigned long long tile = first + i * stride;
+            const unsigned long long t = first + i * stride;
+            const unsigned long long tile = p.reverse ? p.tiles - 1 - t : t;
             const int bi = find_bucket<kMaxBucketsPerLaunch>(p.bk, p.nb, tile);
             const BucketDesc bd = p.bk[bi];
             const unsigned long long base = (tile - bd.tile0) * TILE;
@@ -207,8 +234,13 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                         }
                     }
                     const unsigned long long off = base + (unsigned long long)j * E;
-                    store_floats<SW, E / SW>(bd.theta + off, th);
-                    if (has_v) store_floats<SW, E / SW>(bd.v + off, vv);
+                    if constexpr (WIDE) {
+                        store_floats<SW, E / SW>(bd.theta + off, th);
+                        if (has_v) store_floats<SW, E / SW>(bd.v + off, vv);
+                    } else {
+                        store_floats_policy<E>(bd.theta + off, th, pol_keep);
+                        if (has_v) store_floats_policy<E>(bd.v + off, vv, pol_keep);
+                    }
                     if (has_lp) store_lp<E / 2>(bd.lp + off, th);
                 }
             } else {
