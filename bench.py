@@ -457,7 +457,60 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
             out[key + "+cuda_graph"] = bsp_line(job, gms, 2000, 2000, peak)
             out[key + "+cuda_graph"]["note"] = "50 steps per graph, fixed batches; L2-resident"
             del graph
+            # whole steps (device-side re-batch + fused step with device-resident weights) in a graph
+            measured = torch.tensor(sched[0], dtype=torch.float64, device="cuda")
+            with torch.cuda.stream(side):
+                job.omni.ctl_to_device()
+                job.omni.rebatch_device(measured)
+                job.omni.aggregate_bsp_device_batches(job.buckets, job.cfg.lr, job.cfg.momentum)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(50):
+                    job.omni.rebatch_device(measured)
+                    job.omni.aggregate_bsp_device_batches(job.buckets, job.cfg.lr, job.cfg.momentum)
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            e0.record()
+            for i in range(40):
+                measured.copy_(torch.tensor(sched[i % len(sched)], dtype=torch.float64), non_blocking=False)
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            out[key + "+device_controller_graph"] = bsp_line(job, e0.elapsed_time(e1), 2000, 2000, peak)
+            out[key + "+device_controller_graph"]["launches_per_step"] = 2.0
+            out[key + "+device_controller_graph"]["note"] = ("50 x (one-warp re-batch kernel + fused step reading its "
+                                                             "weights from device memory) per graph, new measurements "
+                                                             "copied in before each replay; L2-resident")
+            del graph
         del job
+        torch.cuda.empty_cache()
+    if not only_asp:
+        # the headline step with the controller on the device: measurements already in device memory, a
+        # one-warp re-batch kernel and the fused step enqueued back to back, no host arithmetic
+        job = BspJob("resnet50_bf16", torch, W, B)
+        _, sched = throughput_schedule(job.cfg, 64, W, torch)
+        dev_sched = [torch.tensor(m, dtype=torch.float64, device="cuda") for m in sched]
+        job.omni.ctl_to_device()
+
+        def dev_run(n):
+            for i in range(n):
+                job.omni.rebatch_device(dev_sched[i % len(dev_sched)])
+                job.omni.aggregate_bsp_device_batches(job.buckets, job.cfg.lr, job.cfg.momentum)
+
+        dev_run(5)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dev_run(500)
+        e1.record()
+        torch.cuda.synchronize()
+        out["resnet50_bf16+device_controller"] = bsp_line(job, e0.elapsed_time(e1), 500, 500, peak)
+        out["resnet50_bf16+device_controller"]["launches_per_step"] = 2.0
+        out["resnet50_bf16+device_controller"]["note"] = "re-batch kernel (1 warp) + fused step per step; GB/s counts the step's bytes over the time of both"
+        job.omni.ctl_from_device()
+        del job, dev_sched
         torch.cuda.empty_cache()
     # asynchronous arrivals: 1000 single-worker gradients with controller feedback
     cfg = W.config("resnet50_asp")

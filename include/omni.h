@@ -193,6 +193,34 @@ int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
                             int32_t worker, int32_t b_used, int32_t tau, const void *const *snapshots, float lr,
                             float weight_decay, void *stream);
 
+/* Device-resident controller: the synchronous re-batch (getBsz of Algorithm 1 for every worker,
+ * Eq. 6a/6b, dead-band Eq. 7, bounds, Eq. 8) as a one-warp kernel on a device copy of the
+ * controller state, so that a whole step -- re-batch from measurements that are already on the
+ * GPU, then aggregate + update with the new weights -- is enqueued (or captured in a CUDA graph)
+ * without a host round trip.  Arithmetic and results are those of omni_rebatch, bit for bit:
+ * single correctly rounded double operations in the same order, then integers.
+ *
+ * omni_ctl_to_device: copies the host controller state (b_k, smoothed times) and the weights
+ *   lambda_k = float(b_k / sum b) to the device copy, allocating it on a context's first call
+ *   (make that call outside stream capture).  Enqueued on `stream`.
+ * omni_rebatch_device: measured_dev = DEVICE double[K] (throughputs, or times with
+ *   OMNI_INPUT_IS_TIME), 8-byte aligned; new_b_dev = DEVICE int32[K] out, or NULL.  Updates the
+ *   device copy's batches, smoothed times and weights.  A measurement that is not finite or not
+ *   positive leaves the device copy untouched and records OMNI_ERR_BAD_MEASUREMENT, which the
+ *   next omni_ctl_from_device returns (once).  The host controller is not touched: host calls
+ *   (omni_rebatch, omni_get_batches, ...) keep seeing the state of the last
+ *   omni_ctl_from_device.
+ * omni_aggregate_bsp_device_batches: omni_aggregate_bsp with the weights the device copy holds
+ *   (no `b` argument; nothing is checked against B on the host).  Always the bulk-copy ring kernel.
+ * omni_ctl_from_device: synchronises `stream`, copies the device copy back into the host
+ *   controller and omni_stats.weight_sum; returns a recorded device re-batch failure, if any.
+ * Errors: NULL, BAD_CONFIG (no device copy yet; or as omni_aggregate_bsp), ALIGN, CUDA. */
+int omni_ctl_to_device(omni_ctx *ctx, void *stream);
+int omni_ctl_from_device(omni_ctx *ctx, void *stream);
+int omni_rebatch_device(omni_ctx *ctx, const double *measured_dev, int32_t *new_b_dev, void *stream);
+int omni_aggregate_bsp_device_batches(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                                      float lr, float momentum, float weight_decay, void *stream);
+
 /* Same step as omni_aggregate_bsp for gradients that arrive in HOST memory (pinned memory gives
  * asynchronous copies).  host_grads: host array of n_buckets*K host pointers, entry [i*K + k] =
  * worker k's gradient for bucket i.  buckets[i].grads must point at K device staging buffers of

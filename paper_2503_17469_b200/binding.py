@@ -28,6 +28,7 @@ EXPORTS = (
     "omni_rebatch", "omni_asp_report", "omni_rebatch_static", "omni_aggregate_bsp",
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
     "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
+    "omni_ctl_to_device", "omni_ctl_from_device", "omni_rebatch_device", "omni_aggregate_bsp_device_batches",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -78,6 +79,10 @@ def lib() -> C.CDLL:
     L.omni_aggregate_bsp_host.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(vp), C.POINTER(i32),
                                           f32, f32, f32, vp, C.POINTER(C.c_double)]
     L.omni_get_stats.argtypes = [vp, C.POINTER(omni_stats), vp]
+    L.omni_ctl_to_device.argtypes = [vp, vp]
+    L.omni_ctl_from_device.argtypes = [vp, vp]
+    L.omni_rebatch_device.argtypes = [vp, vp, vp, vp]
+    L.omni_aggregate_bsp_device_batches.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, f32, f32, f32, vp]
     L.omni_selftest_wait_expiry.argtypes = [vp, vp]
     L.omni_last_cuda_error.argtypes = [vp]
     L.omni_query_launch.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
@@ -296,6 +301,30 @@ class Omni:
         self._check(lib().omni_asp_push_overwrite(self._h, buckets.array, buckets.n_buckets, buckets.dtype, worker,
                                                   b_used, tau, self._ptr_table(snapshots), lr, weight_decay,
                                                   self._stream(stream)))
+
+    # ---- device-resident controller ---------------------------------------------------------
+    def ctl_to_device(self, stream=None) -> None:
+        """Copy the controller state and the weights to the device copy (allocated on first use)."""
+        self._check(lib().omni_ctl_to_device(self._h, self._stream(stream)))
+
+    def ctl_from_device(self, stream=None) -> List[int]:
+        """Synchronise, copy the device copy back into the host controller; returns the batches.
+        Raises the failure a device re-batch recorded (e.g. a non-positive measurement)."""
+        self._check(lib().omni_ctl_from_device(self._h, self._stream(stream)))
+        return self.batches
+
+    def rebatch_device(self, measured, new_b=None, stream=None) -> None:
+        """``measured``: float64 CUDA tensor of K values; ``new_b``: optional int32 CUDA tensor of K."""
+        assert measured.is_cuda and measured.element_size() == 8 and measured.numel() >= self.K
+        assert new_b is None or (new_b.is_cuda and new_b.element_size() == 4 and new_b.numel() >= self.K)
+        self._check(lib().omni_rebatch_device(self._h, C.c_void_p(measured.data_ptr()),
+                                              C.c_void_p(new_b.data_ptr()) if new_b is not None else None,
+                                              self._stream(stream)))
+
+    def aggregate_bsp_device_batches(self, buckets: BucketSet, lr: float, momentum: float = 0.0,
+                                     weight_decay: float = 0.0, stream=None) -> None:
+        self._check(lib().omni_aggregate_bsp_device_batches(self._h, buckets.array, buckets.n_buckets, buckets.dtype,
+                                                            lr, momentum, weight_decay, self._stream(stream)))
 
     def stats(self, stream=None) -> Stats:
         s = omni_stats()

@@ -11,8 +11,10 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libomni.so"
-SOURCES = [CSRC / "omni.cu", CSRC / "bulk_dispatch.cu", CSRC / "noalloc.cu", CSRC / "controller.cpp"]
-HEADERS = [CSRC / "kernels.cuh", CSRC / "tma_kernels.cuh", CSRC / "dispatch.h", CSRC / "controller.h", PKG.parent / "include" / "omni.h"]
+SOURCES = [CSRC / "omni.cu", CSRC / "bulk_dispatch.cu", CSRC / "device_controller.cu", CSRC / "noalloc.cu",
+           CSRC / "controller.cpp"]
+HEADERS = [CSRC / "kernels.cuh", CSRC / "tma_kernels.cuh", CSRC / "dispatch.h", CSRC / "controller.h",
+           CSRC / "device_controller.h", PKG.parent / "include" / "omni.h"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -5,6 +5,22 @@
 namespace omni {
 namespace {
 
+// Diagnostic: one thread waits, with a short limit, on an mbarrier that nothing will ever
+// complete, then records the expiry in the status word exactly as the ring kernel does.  Lets a
+// test (or an operator) see the bounded-wait path end to end without any kernel misbehaving.
+__global__ void expire_wait_kernel(Workspace *ws, unsigned attempts)
+{
+    __shared__ __align__(8) unsigned long long never;
+    if (threadIdx.x == 0) {
+        mbar_init(&never, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        bool done = false;
+        for (unsigned i = 0; i < attempts && !done; ++i) done = mbar_try_wait(&never, 0);
+        if (!done) atomicExch(&ws->status, kStatusTimeout);
+    }
+}
+
+
 template <typename G, int K> KernelInfo bulk_info()
 {
     constexpr TmaShape sh = tma_shape<G>(K);

@@ -174,6 +174,24 @@ int BatchController::report(int32_t worker, int32_t b_used, double measured, int
     return OMNI_OK;
 }
 
+void BatchController::export_state(int32_t *b, double *time, int32_t *seen) const
+{
+    for (int k = 0; k < OMNI_MAX_K; ++k) {
+        b[k] = batch_[k];
+        time[k] = time_[k];
+        seen[k] = seen_[k] ? 1 : 0;
+    }
+}
+
+void BatchController::import_state(const int32_t *b, const double *time, const int32_t *seen)
+{
+    for (int k = 0; k < cfg_.K; ++k) {
+        batch_[k] = b[k];
+        time_[k] = time[k];
+        seen_[k] = seen[k] != 0;
+    }
+}
+
 // Eq. 4a: b_k = c_k / sum(c) * (K b) with K b = B.
 int BatchController::rebatch_static(const double *capacity, int32_t *new_b)
 {

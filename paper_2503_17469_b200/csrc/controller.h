@@ -26,6 +26,10 @@ public:
     int report(int32_t worker, int32_t b_used, double measured, int32_t *new_b_k);
     // Eq. 4a: open-loop split of B by capacity.
     int rebatch_static(const double *capacity, int32_t *new_b);
+    // Whole state (batches, smoothed times, which workers have a time yet), for the copy of the
+    // controller that lives on the device.  Arrays of OMNI_MAX_K entries.
+    void export_state(int32_t *b, double *time, int32_t *seen) const;
+    void import_state(const int32_t *b, const double *time, const int32_t *seen);
 
 private:
     struct Proposal { double real; int32_t rounded; };

@@ -1,0 +1,173 @@
+// The proportional batch-size controller as a one-warp kernel (getBsz of Algorithm 1 for all K
+// workers + the global-batch rule, Eq. 6a/6b/7/8), and the ring-kernel instantiations that read
+// the weights it leaves in device memory.
+//
+// Lane k owns worker k.  Every floating-point step is a single correctly rounded IEEE double
+// operation written as an intrinsic (__dadd_rn, __dmul_rn, __ddiv_rn: never contracted into a
+// multiply-add), and the one sum that depends on order (the mean compute time) is taken by
+// every lane in ascending k, so the integers that come out are the host controller's, bit for
+// bit.  After the single rounding step everything is integer arithmetic on warp votes and
+// shuffles.
+#include <cuda_runtime.h>
+
+#include "device_controller.h"
+#include "dispatch.h"
+#include "tma_kernels.cuh"
+
+namespace omni {
+namespace {
+
+struct CtlConst {
+    int K, B, b_min, b_max, mode;
+    unsigned flags;
+    double deadband, alpha;
+};
+
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ long long warp_sum(long long x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(kFull, x, o);
+    return x;
+}
+__device__ __forceinline__ long long warp_min(long long x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const long long y = __shfl_xor_sync(kFull, x, o);
+        x = y < x ? y : x;
+    }
+    return x;
+}
+
+__global__ void __launch_bounds__(32) rebatch_kernel(DeviceCtl *c, const CtlConst cc, const double *measured, int32_t *new_b)
+{
+    const int k = threadIdx.x;
+    const bool on = k < cc.K;
+
+    // a measurement that is not a positive finite number fails the call; nothing changes
+    const double m = on ? measured[k] : 1.0;
+    if (__any_sync(kFull, on && !(isfinite(m) && m > 0.0))) {
+        if (k == 0) atomicCAS(&c->status, 0, int(OMNI_ERR_BAD_MEASUREMENT));
+        return;
+    }
+    const int32_t b = on ? c->batch[k] : 1;
+    const double bd = double(b);
+    const double lo = double(cc.b_min), hi = double(cc.b_max);
+
+    // Eq. 6a read backwards (t = b / T), then the EWMA of the compute time; the first sample seeds it
+    const double t = (cc.flags & OMNI_INPUT_IS_TIME) ? m : __ddiv_rn(bd, m);
+    double s = t;
+    if (on && c->seen[k]) s = __dadd_rn(__dmul_rn(cc.alpha, t), __dmul_rn(__dsub_rn(1.0, cc.alpha), c->time[k]));
+
+    // mean compute time, summed in ascending k by every lane
+    double total = 0.0;
+    for (int j = 0; j < cc.K; ++j) total = __dadd_rn(total, __shfl_sync(kFull, s, j));
+    const double tbar = __ddiv_rn(total, double(cc.K));
+
+    // getBsz: Eq. 6b, dead-band (Eq. 7), bounds, one rounding to an integer (half up)
+    int32_t n = 0;
+    if (on) {
+        const double throughput = __ddiv_rn(bd, s);
+        const double error = __dsub_rn(s, tbar);
+        const double target = __dsub_rn(bd, __dmul_rn(throughput, error));
+        const double rel = fabs(__ddiv_rn(__dsub_rn(target, bd), target));
+        double chosen = bd;
+        if (rel >= cc.deadband) chosen = target < lo ? lo : target > hi ? hi : target;
+        double r = floor(__dadd_rn(chosen, 0.5));
+        r = r < lo ? lo : r;
+        r = hi < r ? hi : r;
+        n = int32_t(r);
+    }
+
+    // Eq. 8 on integers with bounds: whole rounds of one unit per movable worker, then the last
+    // partial round to the largest batches (lowest index first among equals)
+    if (cc.mode == OMNI_BSP) {
+        long long gap = (long long)cc.B - warp_sum(on ? n : 0);
+        for (int pass = 0; gap != 0; ++pass) {
+            const int dir = gap > 0 ? 1 : -1;
+            const int wall = dir > 0 ? cc.b_max : cc.b_min;
+            const long long room_k = on ? (long long)(wall - n) * dir : 0;   // units until worker k is pinned
+            const bool movable = room_k > 0;
+            const unsigned members = __ballot_sync(kFull, movable);
+            const int count = __popc(members);
+            if (count == 0 || pass > 2 * OMNI_MAX_K + 2) {
+                if (k == 0) atomicCAS(&c->status, 0, int(OMNI_ERR_INFEASIBLE));
+                return;
+            }
+            const long long room = warp_min(movable ? room_k : (long long)0x7fffffffffffffffLL);
+            const long long need = gap * dir;
+            const long long per = need / count;
+            const long long rounds = room < per ? room : per;
+            if (rounds > 0) {
+                if (movable) n += int32_t(dir * rounds);
+                gap -= dir * rounds * count;
+                continue;
+            }
+            int rank = 0;   // movable workers that come before this one: larger batch, or equal batch and lower index
+            for (int j = 0; j < 32; ++j) {
+                const int32_t nj = __shfl_sync(kFull, n, j);
+                if (((members >> j) & 1u) && (nj > n || (nj == n && j < k))) ++rank;
+            }
+            if (movable && rank < need) n += dir;
+            gap = 0;
+        }
+    }
+
+    // commit, then the weights of Eq. 4b for the step that follows
+    const long long sum_b = warp_sum(on ? n : 0);
+    float lam = 0.0f;
+    if (on) {
+        c->batch[k] = n;
+        c->time[k] = s;
+        c->seen[k] = 1;
+        if (new_b) new_b[k] = n;
+        lam = __double2float_rn((cc.flags & OMNI_UNSCALED_MEAN) ? __ddiv_rn(1.0, double(cc.K))
+                                                                  : __ddiv_rn(double(n), double(sum_b)));
+        c->lam[k] = lam;
+    }
+    double wsum = 0.0;
+    for (int j = 0; j < cc.K; ++j) wsum = __dadd_rn(wsum, double(__shfl_sync(kFull, lam, j)));
+    if (k == 0) {
+        c->weight_sum = wsum;
+        c->rebatches += 1u;
+    }
+}
+
+template <typename G, int K> KernelInfo devlam_info()
+{
+    constexpr TmaShape sh = tma_shape<G>(K);
+    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps, false, false, true>),
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K)};
+}
+
+template <typename G> KernelInfo devlam_for(int K)
+{
+    switch (K) {
+#define OMNI_CASE(k) case k: return devlam_info<G, k>();
+        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
+        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
+        OMNI_CASE(17) OMNI_CASE(18) OMNI_CASE(19) OMNI_CASE(20) OMNI_CASE(21) OMNI_CASE(22) OMNI_CASE(23) OMNI_CASE(24)
+        OMNI_CASE(25) OMNI_CASE(26) OMNI_CASE(27) OMNI_CASE(28) OMNI_CASE(29) OMNI_CASE(30) OMNI_CASE(31) OMNI_CASE(32)
+#undef OMNI_CASE
+    }
+    return {};
+}
+
+}  // namespace
+
+KernelInfo bulk_devlam_kernel(int dtype, int K)
+{
+    return dtype == OMNI_BF16 ? devlam_for<__nv_bfloat16>(K) : devlam_for<float>(K);
+}
+
+int launch_device_rebatch(DeviceCtl *ctl, const omni_config &cfg, const double *measured_dev, int32_t *new_b_dev,
+                          void *stream)
+{
+    const CtlConst cc{cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.mode, cfg.flags, cfg.deadband, cfg.ewma_alpha};
+    rebatch_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctl, cc, measured_dev, new_b_dev);
+    return int(cudaGetLastError());
+}
+
+}  // namespace omni

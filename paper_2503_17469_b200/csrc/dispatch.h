@@ -18,6 +18,9 @@ struct KernelInfo {
 // asynchronous apply of M queued arrivals (M = 1: a single arrival; M <= OMNI_MAX_ASP_BATCH).
 KernelInfo bulk_kernel(int dtype, int K);
 KernelInfo bulk_seq_kernel(int dtype, int M);
+// The synchronous ring kernel that reads its K weights from device memory (BspParams::lam_dev),
+// where the device-side controller leaves them (device_controller.cu).
+KernelInfo bulk_devlam_kernel(int dtype, int K);
 // Whether the ring is the better choice for this many streams: its bulk copies must be at least
 // 2 KB each (true for every K up to OMNI_MAX_K with the current ring geometry; 1 KB copies halve
 // the bandwidth).

@@ -55,6 +55,7 @@ struct BspParams {
     int reverse;     // walk the tiles from the last to the first (see omni.cu: alternating sweeps)
     unsigned long long tiles;
     Workspace *ws;
+    const float *lam_dev;  // device copy of the K weights (device-side controller), read instead of lam by the kernels built for it
 };
 
 struct AspParams {

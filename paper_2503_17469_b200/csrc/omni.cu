@@ -6,6 +6,7 @@
 #include <new>
 
 #include "controller.h"
+#include "device_controller.h"
 #include "dispatch.h"
 #include "kernels.cuh"
 
@@ -26,9 +27,12 @@ struct omni_ctx {
     int last_cuda = 0;
     uint64_t launches = 0;
     unsigned sweep = 0;              // calls that walked the parameters so far (parity = sweep direction)
+    omni::DeviceCtl *dctl = nullptr; // device copy of the controller (omni_ctl_to_device), or null
+    omni::DeviceCtl dctl_stage{};    // host staging for its uploads and downloads
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
     omni::LaunchShape bulk_shape[2][OMNI_MAX_K + 1];    // [dtype][K], bulk-copy ring kernel
     omni::LaunchShape bulk_seq_shape[2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][M]
+    omni::LaunchShape bulk_devlam_shape[2][OMNI_MAX_K + 1];       // [dtype][K], ring kernel with device-resident weights
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
     omni::LaunchShape overwrite_shape[2][2];            // [dtype][wide]
     omni::LaunchShape seq_shape[2][2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][wide][M]
@@ -236,14 +240,18 @@ double fill_weights(const omni_ctx *ctx, const int32_t *b, float *lam)
     return wsum;
 }
 
+// lam: the K weights on the host (they travel as kernel parameters), or null with lam_dev: the
+// weights in device memory, which only the ring kernel built for that reads.
 int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t dtype, const float *lam,
-                float lr, float mu, float wd, cudaStream_t stream)
+                const float *lam_dev, float lr, float mu, float wd, cudaStream_t stream)
 {
     const int K = ctx->ctl.K();
-    const bool bulk = use_bulk(ctx, dtype, K);
+    const bool bulk = lam_dev || use_bulk(ctx, dtype, K);
     const bool wide = all_aligned32(buckets, n_buckets, 0, K);
-    const KernelInfo ki = bulk ? bulk_kernel(dtype, K) : bsp_kernel(dtype, K, wide);
-    LaunchShape &shape = bulk ? ctx->bulk_shape[dtype][K] : ctx->bsp_shape[dtype][wide][K];
+    const KernelInfo ki = lam_dev ? bulk_devlam_kernel(dtype, K) : bulk ? bulk_kernel(dtype, K) : bsp_kernel(dtype, K, wide);
+    LaunchShape &shape = lam_dev ? ctx->bulk_devlam_shape[dtype][K]
+                         : bulk  ? ctx->bulk_shape[dtype][K]
+                                 : ctx->bsp_shape[dtype][wide][K];
     int rc = shape_for(ctx, ki, shape);
     if (rc != OMNI_OK) return rc;
     const unsigned long long tile = ki.tile;
@@ -264,7 +272,8 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
             ++nb;
         }
         // an empty call still runs one (empty) launch so that the squared norm reads 0
-        for (int k = 0; k < K; ++k) p.lam[k] = lam[k];
+        for (int k = 0; k < K && lam; ++k) p.lam[k] = lam[k];
+        p.lam_dev = lam_dev;
         p.lr = lr; p.mu = mu; p.wd = wd;
         p.nb = nb;
         p.accumulate = launched > 0;
@@ -327,6 +336,7 @@ void omni_destroy(omni_ctx *ctx)
 {
     if (!ctx) return;
     if (ctx->ws) cudaFree(ctx->ws);
+    if (ctx->dctl) cudaFree(ctx->dctl);
     if (ctx->host_cell) cudaFreeHost(ctx->host_cell);
     delete ctx;
 }
@@ -432,7 +442,7 @@ int omni_aggregate_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buck
     if (rc != OMNI_OK) return rc;
     float lam[OMNI_MAX_K];
     const double wsum = fill_weights(ctx, b, lam);
-    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, lr, momentum, weight_decay,
+    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, nullptr, lr, momentum, weight_decay,
                      static_cast<cudaStream_t>(stream));
     if (rc != OMNI_OK) return rc;
     ctx->tally.weight_sum = wsum;
@@ -463,7 +473,7 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
                                            buckets[i].n * esz, cudaMemcpyHostToDevice, s));
     float lam[OMNI_MAX_K];
     const double wsum = fill_weights(ctx, b, lam);
-    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, lr, momentum, weight_decay, s);
+    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, nullptr, lr, momentum, weight_decay, s);
     if (rc != OMNI_OK) return rc;
     ctx->tally.weight_sum = wsum;
     ctx->tally.steps += 1;
@@ -637,6 +647,73 @@ int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
     ctx->tally.arrivals += 1;
     ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
     if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+    return OMNI_OK;
+}
+
+// ---- device-resident controller ----------------------------------------------------------------
+
+int omni_ctl_to_device(omni_ctx *ctx, void *stream)
+{
+    if (!ctx) return OMNI_ERR_NULL;
+    int rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    if (!ctx->dctl) OMNI_CUDA(ctx, cudaMalloc(&ctx->dctl, sizeof(DeviceCtl)));
+    DeviceCtl &st = ctx->dctl_stage;
+    std::memset(&st, 0, sizeof st);
+    ctx->ctl.export_state(st.batch, st.time, st.seen);
+    st.weight_sum = fill_weights(ctx, st.batch, st.lam);
+    // pageable source: the runtime stages it before the call returns, so `st` may be reused
+    OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->dctl, &st, sizeof st, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)));
+    return OMNI_OK;
+}
+
+int omni_ctl_from_device(omni_ctx *ctx, void *stream)
+{
+    if (!ctx) return OMNI_ERR_NULL;
+    if (!ctx->dctl) return OMNI_ERR_BAD_CONFIG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DeviceCtl &st = ctx->dctl_stage;
+    OMNI_CUDA(ctx, cudaMemcpyAsync(&st, ctx->dctl, sizeof st, cudaMemcpyDeviceToHost, s));
+    OMNI_CUDA(ctx, cudaStreamSynchronize(s));
+    ctx->ctl.import_state(st.batch, st.time, st.seen);
+    ctx->tally.weight_sum = st.weight_sum;
+    if (st.status != 0) {
+        // a device re-batch refused its input since the last read: report it once and clear it
+        OMNI_CUDA(ctx, cudaMemsetAsync(&ctx->dctl->status, 0, sizeof(int32_t), s));
+        return st.status;
+    }
+    return OMNI_OK;
+}
+
+int omni_rebatch_device(omni_ctx *ctx, const double *measured_dev, int32_t *new_b_dev, void *stream)
+{
+    if (!ctx || !measured_dev) return OMNI_ERR_NULL;
+    if (!ctx->dctl) return OMNI_ERR_BAD_CONFIG;
+    if ((reinterpret_cast<uintptr_t>(measured_dev) & 7u) || (reinterpret_cast<uintptr_t>(new_b_dev) & 3u)) return OMNI_ERR_ALIGN;
+    int rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    const int e = launch_device_rebatch(ctx->dctl, ctx->ctl.config(), measured_dev, new_b_dev, stream);
+    if (e != 0) {
+        ctx->last_cuda = e;
+        return OMNI_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return OMNI_OK;
+}
+
+int omni_aggregate_bsp_device_batches(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                                      float lr, float momentum, float weight_decay, void *stream)
+{
+    if (!ctx) return OMNI_ERR_NULL;
+    if (!ctx->dctl) return OMNI_ERR_BAD_CONFIG;
+    int rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, -1, momentum);
+    if (rc != OMNI_OK) return rc;
+    rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, nullptr, ctx->dctl->lam, lr, momentum, weight_decay,
+                     static_cast<cudaStream_t>(stream));
+    if (rc != OMNI_OK) return rc;
+    ctx->tally.steps += 1;
     return OMNI_OK;
 }
 

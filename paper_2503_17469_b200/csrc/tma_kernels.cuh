@@ -105,7 +105,7 @@ template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int 
     return unsigned(s.stages) * unsigned(s.tile) * unsigned(K * int(sizeof(G)) + 8);
 }
 
-template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false>
+template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false, bool DEVLAM = false>
 __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_constant__ BspParams p)
 {
     constexpr int THREADS = (NCW + 1) * 32;
@@ -137,6 +137,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
     if (warp == NCW) {
         // ---------------- producer warp: lane 0 issues the copies ----------------
         if (lane == 0) {
+            unsigned long long armed = 0;          // stages armed so far (= issue index of the next one)
             for (unsigned long long i = 0; i < mine; ++i) {
                 const int s = int(i % STAGES);
                 const unsigned long long t = first + i * stride;
@@ -148,6 +149,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                     atomicExch(&p.ws->status, kStatusTimeout);
                     break;
                 }
+                armed = i + 1;
                 if (base + TILE > bd.n) {          // ragged tile: consumers read it from global memory
                     mbar_arrive(&full[s]);
                     continue;
@@ -159,9 +161,28 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                 bulk_load(st + K * GB, bd.theta + base, FB, &full[s], pol_keep);
                 if (with_v) bulk_load(st + K * GB + FB, bd.v + base, FB, &full[s], pol_keep);
             }
+            // Leave no copy in flight when this CTA gives its shared memory back: the stages armed
+            // last must have landed.  After a normal run the consumers have already seen them
+            // land, so this returns at once; it matters when a wait above or below gave up.
+            for (unsigned long long j = armed > STAGES ? armed - STAGES : 0; j < armed; ++j)
+                if (!mbar_wait(&full[j % STAGES], unsigned((j / STAGES) & 1))) {
+                    atomicExch(&p.ws->status, kStatusTimeout);
+                    break;
+                }
         }
     } else {
         // ---------------- consumer warps ----------------
+        // DEVLAM: the weights come from device memory (written by the device-side controller)
+        // instead of the kernel parameters.
+        float lamr[DEVLAM ? K : 1];
+        if constexpr (DEVLAM) {
+#pragma unroll
+            for (int k = 0; k < K; ++k) lamr[k] = __ldcg(p.lam_dev + k);
+        }
+        auto weight = [&](int k) -> float {
+            if constexpr (DEVLAM) return lamr[k];
+            else return p.lam[k];
+        };
         for (unsigned long long i = 0; i < mine; ++i) {
             const int s = int(i % STAGES);
             const unsigned long long t = first + i * stride;
@@ -193,7 +214,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                     if constexpr (SEQ) {
 #pragma unroll
                         for (int k = 0; k < K; ++k) {
-                            const float eta = p.lam[k];
+                            const float eta = weight(k);
 #pragma unroll
                             for (int h = 0; h < NV; ++h) {
                                 const uint4 r = *reinterpret_cast<const uint4 *>(st + k * GB + size_t(j * NV + h) * 16);
@@ -211,7 +232,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                         for (int e = 0; e < E; ++e) acc[e] = 0.0f;
 #pragma unroll
                         for (int k = 0; k < K; ++k) {
-                            const float lam = p.lam[k];
+                            const float lam = weight(k);
 #pragma unroll
                             for (int h = 0; h < NV; ++h) {
                                 const uint4 r = *reinterpret_cast<const uint4 *>(st + k * GB + size_t(j * NV + h) * 16);
@@ -259,7 +280,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                                 float gk[V];
                                 widen<G, 4>(raw[k], gk);
 #pragma unroll
-                                for (int e = 0; e < V; ++e) th[e] = update_one(gk[e], th[e], vv[e], p.lam[k], mu, wd);
+                                for (int e = 0; e < V; ++e) th[e] = update_one(gk[e], th[e], vv[e], weight(k), mu, wd);
                             }
                         } else {
                             float acc[V];
@@ -269,7 +290,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                             for (int k = 0; k < K; ++k) {
                                 float gk[V];
                                 widen<G, 4>(raw[k], gk);
-                                const float lam = p.lam[k];
+                                const float lam = weight(k);
 #pragma unroll
                                 for (int e = 0; e < V; ++e) acc[e] = __fmaf_rn(lam, gk[e], acc[e]);
                             }
@@ -291,12 +312,12 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                             if constexpr (SEQ) {
 #pragma unroll
                                 for (int k = 0; k < K; ++k)
-                                    t = update_one(widen1<G>(static_cast<const G *>(p.g[bi][k]), j), t, vj, p.lam[k], mu, wd);
+                                    t = update_one(widen1<G>(static_cast<const G *>(p.g[bi][k]), j), t, vj, weight(k), mu, wd);
                             } else {
                                 float acc = 0.0f;
 #pragma unroll
                                 for (int k = 0; k < K; ++k)
-                                    acc = __fmaf_rn(p.lam[k], widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
+                                    acc = __fmaf_rn(weight(k), widen1<G>(static_cast<const G *>(p.g[bi][k]), j), acc);
                                 t = update_one(acc, t, vj, lr, mu, wd);
                                 sq += (double)(acc * acc);
                             }
@@ -313,21 +334,6 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
         }
     }
     if constexpr (!SEQ) finish_sqnorm<THREADS>(sq, p.ws, p.accumulate);
-}
-
-// Diagnostic: one thread waits, with a short limit, on an mbarrier that nothing will ever
-// complete, then records the expiry in the status word exactly as the ring kernel does.  Lets a
-// test (or an operator) see the bounded-wait path end to end without any kernel misbehaving.
-__global__ void expire_wait_kernel(Workspace *ws, unsigned attempts)
-{
-    __shared__ __align__(8) unsigned long long never;
-    if (threadIdx.x == 0) {
-        mbar_init(&never, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        bool done = false;
-        for (unsigned i = 0; i < attempts && !done; ++i) done = mbar_try_wait(&never, 0);
-        if (!done) atomicExch(&ws->status, kStatusTimeout);
-    }
 }
 
 }  // namespace omni
