@@ -166,6 +166,14 @@ def test_argument_validation_happens_before_any_cuda_call():
     assert asp(2, 32, 0, 0.1, 0.0, 0.0, None) == B.ERR_BAD_WORKER
     assert asp(0, 0, 0, 0.1, 0.0, 0.0, None) == B.ERR_BAD_BATCH
     assert asp(0, 32, -1, 0.1, 0.0, 0.0, None) == B.ERR_BAD_TAU
+    # the device-resident controller: nothing works before the device copy exists
+    assert L.omni_ctl_to_device(None, None) == B.ERR_NULL
+    assert L.omni_ctl_from_device(None, None) == B.ERR_NULL
+    assert L.omni_ctl_from_device(o._h, None) == B.ERR_BAD_CONFIG
+    assert L.omni_rebatch_device(o._h, None, None, None) == B.ERR_NULL
+    assert L.omni_rebatch_device(o._h, 0x1000, None, None) == B.ERR_BAD_CONFIG
+    assert L.omni_aggregate_bsp_device_batches(None, bk, 1, 0, 0.1, 0.9, 0.0, None) == B.ERR_NULL
+    assert L.omni_aggregate_bsp_device_batches(o._h, bk, 1, 0, 0.1, 0.9, 0.0, None) == B.ERR_BAD_CONFIG
     assert o.kernel_launches == 0
     s = o.stats()
     assert s.steps == 0 and s.arrivals == 0 and sum(s.tau_hist) == 0
