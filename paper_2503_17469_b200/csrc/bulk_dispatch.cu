@@ -43,9 +43,9 @@ template <typename G> KernelInfo bulk_for(int K)
 
 template <typename G, int M> KernelInfo bulk_seq_info()
 {
-    constexpr TmaShape sh = tma_shape<G>(M);
+    constexpr TmaShape sh = tma_seq_shape<G>(M);
     return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, M, sh.tile, sh.stages, sh.consumer_warps, false, true>),
-            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(M)};
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_ring_bytes(sh, M, int(sizeof(G)))};
 }
 
 template <typename G> KernelInfo bulk_seq_for(int M)

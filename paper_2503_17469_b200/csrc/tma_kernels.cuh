@@ -86,23 +86,40 @@ struct TmaShape { int tile, stages, consumer_warps; };
 // bulk copy (4 KB or more per gradient stream is as fast as the register kernel, 2 KB costs
 // 2-3 %, 1 KB halves the bandwidth) and about 150 KB in flight per SM; more stages do not help.
 // So: the largest tile whose stage stays within 80 KB, and as many stages as make ~150 KB
-// (halving the stage size or a 110 KB ring cost 3-5 % in back-to-back runs).  Eight consumer
+// (halving the stage size or a 110 KB ring cost 3-5 % in back-to-back runs; with 4 KB copies a
+// larger ring loses 1-4 %).  Where that rule leaves copies of 2 KB (float K > 18, bfloat16
+// K > 16), a tile of one and a half times the size -- 3 KB copies, two stages of up to 108 KB --
+// wins 2-4 % (float K = 24: 7.10 vs 6.95 TB/s, K = 32: 6.93 vs 6.68; bfloat16 K = 32: 6.85 vs
+// 6.63), while 4 KB copies in a 213 KB ring lose again (float K = 24: 6.88).  Eight consumer
 // warps: 4 were 1-3 % slower, 6-12 the same, 16 slower again on bf16.
 template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
 {
     const int per_elem = K * int(sizeof(G)) + 8;
     int tile = 4096;
     while (tile > 256 && tile * per_elem > 80 * 1024) tile /= 2;
+    if (tile * int(sizeof(G)) < 4096 && 2 * (tile * 3 / 2) * per_elem <= 216 * 1024) tile = tile * 3 / 2;
     const int stage = tile * per_elem;
     int stages = (152 * 1024 + stage / 2) / stage;
     if (stages < 2) stages = 2;
     if (stages > 8) stages = 8;
     return {tile, stages, 8};
 }
+// The asynchronous apply of M queued arrivals uses the same geometry with M streams, except the
+// single float arrival: with most of theta coming from L2 (see the alternating sweeps in
+// omni.cu) it is no longer DRAM-bound, and four stages with sixteen consumer warps gain 3 %
+// (8.20 vs 7.96 TB/s algorithmic).
+template <typename G> __host__ __device__ constexpr TmaShape tma_seq_shape(int M)
+{
+    if (M == 1 && sizeof(G) == 4) return {4096, 4, 16};
+    return tma_shape<G>(M);
+}
+__host__ __device__ constexpr unsigned tma_ring_bytes(TmaShape s, int streams, int gsize)
+{
+    return unsigned(s.stages) * unsigned(s.tile) * unsigned(streams * gsize + 8);
+}
 template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int K)
 {
-    const TmaShape s = tma_shape<G>(K);
-    return unsigned(s.stages) * unsigned(s.tile) * unsigned(K * int(sizeof(G)) + 8);
+    return tma_ring_bytes(tma_shape<G>(K), K, int(sizeof(G)));
 }
 
 template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false, bool DEVLAM = false>
