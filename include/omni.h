@@ -64,7 +64,8 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
  * every call as well (and serve omni_aggregate_bsp_noalloc and omni_asp_push_overwrite).  The ring
  * kernels also alternate the direction in which successive calls walk the parameters and keep
  * theta and v in L2 with evict-last priority, so that a call finds the part its predecessor
- * touched last still in cache.  The two flags force
+ * touched last still in cache, and are launched with programmatic stream serialization (they
+ * wait for the previous launch themselves, after their set-up).  The two flags force
  * one family; results are the same bit for bit.  A bounded wait of the ring that runs out
  * surfaces as OMNI_ERR_TIMEOUT from omni_get_stats. */
 #define OMNI_BULK_COPY 8u

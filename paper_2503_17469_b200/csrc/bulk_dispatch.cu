@@ -25,7 +25,7 @@ template <typename G, int K> KernelInfo bulk_info()
 {
     constexpr TmaShape sh = tma_shape<G>(K);
     return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps, false>),
-            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K)};
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K), true};
 }
 
 template <typename G> KernelInfo bulk_for(int K)
@@ -45,7 +45,7 @@ template <typename G, int M> KernelInfo bulk_seq_info()
 {
     constexpr TmaShape sh = tma_seq_shape<G>(M);
     return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, M, sh.tile, sh.stages, sh.consumer_warps, false, true>),
-            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_ring_bytes(sh, M, int(sizeof(G)))};
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_ring_bytes(sh, M, int(sizeof(G))), true};
 }
 
 template <typename G> KernelInfo bulk_seq_for(int M)

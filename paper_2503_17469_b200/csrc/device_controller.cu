@@ -139,7 +139,7 @@ template <typename G, int K> KernelInfo devlam_info()
 {
     constexpr TmaShape sh = tma_shape<G>(K);
     return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps, false, false, true>),
-            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K)};
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K), true};
 }
 
 template <typename G> KernelInfo devlam_for(int K)

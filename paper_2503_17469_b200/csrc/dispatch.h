@@ -12,6 +12,8 @@ struct KernelInfo {
     int ctas_per_sm = 0;          // wanted CTAs per SM (capped by what fits)
     unsigned long long tile = 0;  // elements per tile
     unsigned smem = 0;            // dynamic shared memory per CTA, bytes
+    bool dependent_launch = false;  // the kernel waits for its predecessor itself (griddepcontrol.wait): launch it
+                                    // with programmatic stream serialization so that its set-up overlaps that tail
 };
 
 // Bulk-copy ring kernels (bulk_dispatch.cu): the synchronous step for K workers, and the

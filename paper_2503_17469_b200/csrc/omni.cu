@@ -220,6 +220,22 @@ int check_buckets(const omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buc
 int launch(omni_ctx *ctx, const KernelInfo &ki, int grid, void *params, cudaStream_t stream)
 {
     void *args[] = {params};
+    if (ki.dependent_launch) {
+        // the ring kernels order themselves after the previous launch (see tma_kernels.cuh)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(ki.threads);
+        cfg.dynamicSmemBytes = ki.smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        OMNI_CUDA(ctx, cudaLaunchKernelExC(&cfg, ki.fn, args));
+        ctx->launches += 1;
+        return OMNI_OK;
+    }
     OMNI_CUDA(ctx, cudaLaunchKernel(ki.fn, dim3(grid), dim3(ki.threads), args, ki.smem, stream));
     ctx->launches += 1;
     return OMNI_OK;

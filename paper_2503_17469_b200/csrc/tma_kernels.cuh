@@ -149,6 +149,13 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Programmatic dependent launch (the host launches this kernel with stream serialization
+    // relaxed): let the next launch of the stream take this SM as soon as this CTA leaves it, and
+    // do not touch global memory before the previous launch has finished and its writes are
+    // visible.  Everything above is set-up that may overlap the predecessor's tail.  Without
+    // the launch attribute both instructions do nothing.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     double sq = 0.0;
     if (warp == NCW) {
