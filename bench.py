@@ -388,6 +388,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(HEADLINE, 12.0, torch, W)
 
+    traffic = recorded_traffic("bsp_tma_bf16_k16" if block == 288 else "bsp_fused_bf16_k16")
     if rank == 0:
         line = {
             "metric": METRIC, "value": world * line_main["params_per_s"], "unit": UNIT, "n_gpus": world,
@@ -404,7 +405,10 @@ def main():
                          "frac": line_main["frac_of_measured"], "peak_source": f"of {peak_kind}",
                          "kernel": "bsp_tma_kernel<bf16,16,tile 2048,2 stages>" if block == 288 else "bsp_fused_kernel<bf16,16>", "bytes_per_launch": job.bytes_per_step,
                          "note": "algorithmic bytes; part of theta/v is re-used from L2 between launches, so DRAM traffic per launch is lower (see traffic) and the fraction can exceed 1",
-                         "traffic": recorded_traffic("bsp_tma_bf16_k16" if block == 288 else "bsp_fused_bf16_k16")},
+                         "traffic": traffic,
+                         # what DRAM actually served per second: the ncu traffic per launch over this run's launch time
+                         "dram_gbs": (traffic / (ms * 1e-3 / max(launches, 1)) / 1e9) if traffic else None,
+                         "dram_frac": (traffic / (ms * 1e-3 / max(launches, 1)) / 1e9 / peak) if traffic else None},
             "e2e": {"value": world * cfg.P * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": 8, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": launches,

@@ -215,12 +215,30 @@ int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
  *   (no `b` argument; nothing is checked against B on the host).  Always the bulk-copy ring kernel.
  * omni_ctl_from_device: synchronises `stream`, copies the device copy back into the host
  *   controller and omni_stats.weight_sum; returns a recorded device re-batch failure, if any.
+ * omni_ctl_to_device and omni_ctl_from_device copy between pageable host memory and the device and
+ * are not meant to be captured; omni_rebatch_device and omni_aggregate_bsp_device_batches are
+ * plain kernel launches.
  * Errors: NULL, BAD_CONFIG (no device copy yet; or as omni_aggregate_bsp), ALIGN, CUDA. */
 int omni_ctl_to_device(omni_ctx *ctx, void *stream);
 int omni_ctl_from_device(omni_ctx *ctx, void *stream);
 int omni_rebatch_device(omni_ctx *ctx, const double *measured_dev, int32_t *new_b_dev, void *stream);
 int omni_aggregate_bsp_device_batches(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                                       float lr, float momentum, float weight_decay, void *stream);
+
+/* Parameter-range sharding for one rank per GPU (no counterpart in the paper, whose workers
+ * all-reduce whole gradients; this is the reduce-scatter form of the same sum).  Every element of
+ * the step is independent of every other, so the AllReduce of Algorithm 1 followed by the update
+ * can run as: rank r owns the elements [begin, begin + count) of each bucket, reads that range of
+ * all K workers' gradients (its own locally, the others through peer-mapped pointers placed in
+ * omni_bucket.grads), runs omni_aggregate_bsp on the sub-range, and the ranks then exchange the
+ * updated ranges (all-gather) and add their squared norms.  This call only computes the range:
+ * n elements are cut into units of OMNI_SHARD_UNIT elements (so that every range starts on a
+ * 256-byte boundary of a float buffer and a 128-byte boundary of a bfloat16 buffer) and the
+ * units are dealt out contiguously, rank counts differing by at most one unit; the ranges of
+ * ranks 0..world-1 tile [0, n) in order.  count may be 0 when n is small.
+ * Errors: NULL, BAD_CONFIG (world < 1, rank outside 0..world-1). */
+#define OMNI_SHARD_UNIT 64
+int omni_shard_range(uint64_t n, int32_t world, int32_t rank, uint64_t *begin, uint64_t *count);
 
 /* Same step as omni_aggregate_bsp for gradients that arrive in HOST memory (pinned memory gives
  * asynchronous copies).  host_grads: host array of n_buckets*K host pointers, entry [i*K + k] =

@@ -29,6 +29,7 @@ EXPORTS = (
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
     "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
     "omni_ctl_to_device", "omni_ctl_from_device", "omni_rebatch_device", "omni_aggregate_bsp_device_batches",
+    "omni_shard_range",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -83,6 +84,7 @@ def lib() -> C.CDLL:
     L.omni_ctl_from_device.argtypes = [vp, vp]
     L.omni_rebatch_device.argtypes = [vp, vp, vp, vp]
     L.omni_aggregate_bsp_device_batches.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, f32, f32, f32, vp]
+    L.omni_shard_range.argtypes = [C.c_uint64, i32, i32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.omni_selftest_wait_expiry.argtypes = [vp, vp]
     L.omni_last_cuda_error.argtypes = [vp]
     L.omni_query_launch.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
@@ -92,6 +94,15 @@ def lib() -> C.CDLL:
                                              f32, f32, f32, vp, vp]
     _lib = L
     return L
+
+
+def shard_range(n: int, world: int, rank: int):
+    """(begin, count) of the elements of an n-element bucket that rank ``rank`` of ``world`` owns."""
+    b, c = C.c_uint64(), C.c_uint64()
+    rc = lib().omni_shard_range(n, world, rank, C.byref(b), C.byref(c))
+    if rc != OK:
+        raise OmniError(rc)
+    return b.value, c.value
 
 
 class OmniError(RuntimeError):
