@@ -550,6 +550,52 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
                            "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_param": cfg.bytes_per_param(),
                            "launches_per_arrival": (o.kernel_launches - l0) / cfg.steps, "tau_max": st.tau_max,
                            "tau_hist_0_31_overflow": st.tau_hist}
+    # Algorithm 2 taken literally on the same stream: the arriving worker's local step overwrites the server
+    # copy (push), then the worker reads the new parameters back into its snapshot (pull)
+    snaps = [torch.empty_like(buf.theta) for _ in range(cfg.K)]
+    o3 = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.ASP)
+    snap_views = [[sn[bk.start:bk.start + bk.n] for bk in buf.layout.buckets] for sn in snaps]
+    for k in range(cfg.K):
+        o3.asp_pull(bs, snap_views[k])
+    b = [cfg.global_batch // cfg.K] * cfg.K
+    last = [0] * cfg.K
+
+    def literal(i0, n):
+        for i in range(i0, i0 + n):
+            k = W.pick_worker(u[i], [T[j] / b[j] for j in range(cfg.K)])
+            o3.asp_push_overwrite(bs, k, b[k], i - last[k], snap_views[k], cfg.lr)
+            o3.asp_pull(bs, snap_views[k])
+            last[k] = i + 1
+            b[k] = o3.asp_report(k, b[k], T[k])
+
+    def fused(i0, n):
+        for i in range(i0, i0 + n):
+            k = W.pick_worker(u[i], [T[j] / b[j] for j in range(cfg.K)])
+            o3.asp_push_pull(bs, k, b[k], i - last[k], snap_views[k], cfg.lr)
+            last[k] = i + 1
+            b[k] = o3.asp_report(k, b[k], T[k])
+
+    for key, fn, bpp, note in (
+            ("resnet50_asp_push_overwrite+pull", literal, 20,
+             "per arrival: push (read snapshot + gradient, write theta: 12 B/param) + pull (device copies theta -> "
+             "snapshot: 8 B/param)"),
+            ("resnet50_asp_push_pull_fused", fused, 16,
+             "per arrival: one pass reads snapshot + gradient and writes theta and the snapshot")):
+        b[:] = [cfg.global_batch // cfg.K] * cfg.K
+        last[:] = [0] * cfg.K
+        fn(0, 50)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn(50, cfg.steps)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        gbs = bpp * cfg.P * cfg.steps / (ms * 1e-3) / 1e9
+        out[key] = {"params_per_s": cfg.P * cfg.steps / (ms * 1e-3), "ms_per_arrival": ms / cfg.steps,
+                    "achieved_gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+                    "bytes_per_param": bpp, "note": note}
+    del snaps, snap_views, o3
     # the same stream with arrivals queued four at a time and applied in one pass each
     m = 4
     b = [cfg.global_batch // cfg.K] * cfg.K

@@ -61,7 +61,7 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
 #define OMNI_INPUT_IS_TIME 4u   /* measurements are compute times t_k instead of throughputs T_k */
 /* Kernel family.  By default the device calls stage their inputs through shared memory with
  * bulk (TMA) copies and an mbarrier ring; register-staged 128/256-bit-load kernels exist for
- * every call as well (and serve omni_aggregate_bsp_noalloc and omni_asp_push_overwrite).  The ring
+ * every call as well (and serve omni_aggregate_bsp_noalloc).  The ring
  * kernels also alternate the direction in which successive calls walk the parameters and keep
  * theta and v in L2 with evict-last priority, so that a call finds the part its predecessor
  * touched last still in cache, and are launched with programmatic stream serialization (they
@@ -188,11 +188,19 @@ int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_bu
  * (the paper's "overridden" updates), so here the staleness tau changes the result, although it
  * still enters no formula; it is tallied as in omni_apply_asp.  Plain SGD as in Algorithm 2 (no
  * momentum buffer is read or written).  With tau = 0 the result equals omni_apply_asp's.
+ * omni_asp_push_pull: the push above followed at once by the same worker's next pull, as in the
+ * worker loop of Algorithm 2 (pushToPS at the end of one iteration, pullFromPS at the start of the
+ * next), in the same launch: the server copy AND the worker's snapshot receive the new
+ * parameters (snapshots are read and written).  Same result as omni_asp_push_overwrite followed
+ * by omni_asp_pull of that worker, at 16 instead of 20 bytes per parameter.
  * Errors: NULL, BAD_WORKER, BAD_BATCH, BAD_TAU, ALIGN, BAD_CONFIG, CUDA. */
 int omni_asp_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, void *const *snapshots, void *stream);
 int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                             int32_t worker, int32_t b_used, int32_t tau, const void *const *snapshots, float lr,
                             float weight_decay, void *stream);
+int omni_asp_push_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                       int32_t worker, int32_t b_used, int32_t tau, void *const *snapshots, float lr,
+                       float weight_decay, void *stream);
 
 /* Device-resident controller: the synchronous re-batch (getBsz of Algorithm 1 for every worker,
  * Eq. 6a/6b, dead-band Eq. 7, bounds, Eq. 8) as a one-warp kernel on a device copy of the

@@ -29,7 +29,7 @@ EXPORTS = (
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
     "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
     "omni_ctl_to_device", "omni_ctl_from_device", "omni_rebatch_device", "omni_aggregate_bsp_device_batches",
-    "omni_shard_range",
+    "omni_shard_range", "omni_asp_push_pull",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
                                        C.POINTER(i32), f32, f32, f32, vp]
     L.omni_asp_pull.argtypes = [vp, C.POINTER(omni_bucket), i32, C.POINTER(vp), vp]
     L.omni_asp_push_overwrite.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, C.POINTER(vp), f32, f32, vp]
+    L.omni_asp_push_pull.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, C.POINTER(vp), f32, f32, vp]
     L.omni_aggregate_bsp_host.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(vp), C.POINTER(i32),
                                           f32, f32, f32, vp, C.POINTER(C.c_double)]
     L.omni_get_stats.argtypes = [vp, C.POINTER(omni_stats), vp]
@@ -336,6 +337,14 @@ class Omni:
                                      weight_decay: float = 0.0, stream=None) -> None:
         self._check(lib().omni_aggregate_bsp_device_batches(self._h, buckets.array, buckets.n_buckets, buckets.dtype,
                                                             lr, momentum, weight_decay, self._stream(stream)))
+
+    def asp_push_pull(self, buckets: BucketSet, worker: int, b_used: int, tau: int, snapshots: Sequence,
+                      lr: float, weight_decay: float = 0.0, stream=None) -> None:
+        """Push with overwrite and the same worker's next pull in one launch: the server parameters
+        and ``snapshots`` both receive snapshot - eta_k * gradient."""
+        self._check(lib().omni_asp_push_pull(self._h, buckets.array, buckets.n_buckets, buckets.dtype, worker,
+                                             b_used, tau, self._ptr_table(snapshots), lr, weight_decay,
+                                             self._stream(stream)))
 
     def stats(self, stream=None) -> Stats:
         s = omni_stats()

@@ -59,7 +59,19 @@ template <typename G> KernelInfo bulk_seq_for(int M)
     return {};
 }
 
+template <typename G> KernelInfo bulk_overwrite_info()
+{
+    constexpr TmaShape sh = tma_seq_shape<G>(1);
+    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, 1, sh.tile, sh.stages, sh.consumer_warps, false, true, false, true>),
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_ring_bytes(sh, 1, int(sizeof(G))), true};
+}
+
 }  // namespace
+
+KernelInfo bulk_overwrite_kernel(int dtype)
+{
+    return dtype == OMNI_BF16 ? bulk_overwrite_info<__nv_bfloat16>() : bulk_overwrite_info<float>();
+}
 
 KernelInfo bulk_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bulk_for<__nv_bfloat16>(K) : bulk_for<float>(K); }
 KernelInfo bulk_seq_kernel(int dtype, int M) { return dtype == OMNI_BF16 ? bulk_seq_for<__nv_bfloat16>(M) : bulk_seq_for<float>(M); }

@@ -23,6 +23,9 @@ KernelInfo bulk_seq_kernel(int dtype, int M);
 // The synchronous ring kernel that reads its K weights from device memory (BspParams::lam_dev),
 // where the device-side controller leaves them (device_controller.cu).
 KernelInfo bulk_devlam_kernel(int dtype, int K);
+// The ring kernel as push with overwrite (Algorithm 2): one gradient stream, the snapshot in
+// place of theta (BspParams::src), optional copy of the result back to the snapshot (::copy).
+KernelInfo bulk_overwrite_kernel(int dtype);
 // Whether the ring is the better choice for this many streams: its bulk copies must be at least
 // 2 KB each (true for every K up to OMNI_MAX_K with the current ring geometry; 1 KB copies halve
 // the bandwidth).

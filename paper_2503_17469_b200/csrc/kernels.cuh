@@ -56,6 +56,10 @@ struct BspParams {
     unsigned long long tiles;
     Workspace *ws;
     const float *lam_dev;  // device copy of the K weights (device-side controller), read instead of lam by the kernels built for it
+    // push with overwrite on the ring (Algorithm 2): per bucket the snapshot the worker pulled
+    // (read in place of theta) and, if the worker pulls again at once, where the result is copied
+    const float *src[kMaxBucketsPerLaunch];
+    float *copy[kMaxBucketsPerLaunch];
 };
 
 struct AspParams {

@@ -35,6 +35,7 @@ struct omni_ctx {
     omni::LaunchShape bulk_devlam_shape[2][OMNI_MAX_K + 1];       // [dtype][K], ring kernel with device-resident weights
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
     omni::LaunchShape overwrite_shape[2][2];            // [dtype][wide]
+    omni::LaunchShape bulk_overwrite_shape[2];          // [dtype], ring kernel as push with overwrite
     omni::LaunchShape seq_shape[2][2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][wide][M]
 };
 
@@ -608,9 +609,11 @@ int omni_asp_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, 
     return OMNI_OK;
 }
 
-int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
-                            int32_t worker, int32_t b_used, int32_t tau, const void *const *snapshots, float lr,
-                            float weight_decay, void *stream)
+// Algorithm 2's worker step + pushToPS (and, with write_back, the pullFromPS that follows it) in
+// one launch: ring kernel by default, register kernel on a context that forces that family.
+static int push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                          int32_t worker, int32_t b_used, int32_t tau, void *const *snapshots, bool write_back,
+                          float lr, float weight_decay, void *stream)
 {
     if (!ctx) return OMNI_ERR_NULL;
     const int K = ctx->ctl.K();
@@ -632,38 +635,95 @@ int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
     const double eta_k = (ctx->ctl.config().flags & OMNI_ASP_NO_LR_SCALE)
                              ? double(lr)
                              : double(lr) * double(b_used) / double(ctx->ctl.B());
-    const KernelInfo ki = overwrite_kernel(grad_dtype, wide);
-    LaunchShape &shape = ctx->overwrite_shape[grad_dtype][wide];
-    rc = shape_for(ctx, ki, shape);
-    if (rc != OMNI_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    OverwriteParams p;
-    int i = 0;
-    while (i < n_buckets) {
-        std::memset(&p, 0, sizeof p);
-        unsigned long long tiles = 0;
-        int nb = 0;
-        for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
-            const omni_bucket &bk = buckets[i];
-            if (bk.n == 0) continue;
-            p.bk[nb] = {static_cast<float *>(bk.param), nullptr, static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
-            p.g[nb] = bk.grads[worker];
-            p.snap[nb] = static_cast<const float *>(snapshots[i]);
-            tiles += (bk.n + ki.tile - 1) / ki.tile;
-            ++nb;
-        }
-        if (nb == 0) break;
-        p.eta = float(eta_k); p.wd = weight_decay;
-        p.nb = nb;
-        p.tiles = tiles;
-        const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
-        rc = launch(ctx, ki, grid, &p, static_cast<cudaStream_t>(stream));
+    if (use_bulk(ctx, grad_dtype, 1)) {
+        const KernelInfo ki = bulk_overwrite_kernel(grad_dtype);
+        LaunchShape &shape = ctx->bulk_overwrite_shape[grad_dtype];
+        rc = shape_for(ctx, ki, shape);
         if (rc != OMNI_OK) return rc;
+        BspParams p;
+        int i = 0;
+        while (i < n_buckets) {
+            std::memset(&p, 0, sizeof p);
+            unsigned long long tiles = 0;
+            int nb = 0;
+            for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+                const omni_bucket &bk = buckets[i];
+                if (bk.n == 0) continue;
+                p.bk[nb] = {static_cast<float *>(bk.param), nullptr, static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
+                p.g[nb][0] = bk.grads[worker];
+                p.src[nb] = static_cast<const float *>(snapshots[i]);
+                p.copy[nb] = write_back ? static_cast<float *>(snapshots[i]) : nullptr;
+                tiles += (bk.n + ki.tile - 1) / ki.tile;
+                ++nb;
+            }
+            if (nb == 0) break;
+            p.lam[0] = float(eta_k);
+            p.wd = weight_decay;
+            p.nb = nb;
+            p.reverse = int(ctx->sweep & 1u);
+            p.tiles = tiles;
+            p.ws = ctx->ws;
+            const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
+            rc = launch(ctx, ki, grid, &p, s);
+            if (rc != OMNI_OK) return rc;
+        }
+        ctx->sweep += 1;
+    } else {
+        const KernelInfo ki = overwrite_kernel(grad_dtype, wide);
+        LaunchShape &shape = ctx->overwrite_shape[grad_dtype][wide];
+        rc = shape_for(ctx, ki, shape);
+        if (rc != OMNI_OK) return rc;
+        OverwriteParams p;
+        int i = 0;
+        while (i < n_buckets) {
+            std::memset(&p, 0, sizeof p);
+            unsigned long long tiles = 0;
+            int nb = 0;
+            for (; i < n_buckets && nb < kMaxBucketsPerLaunch; ++i) {
+                const omni_bucket &bk = buckets[i];
+                if (bk.n == 0) continue;
+                p.bk[nb] = {static_cast<float *>(bk.param), nullptr, static_cast<__nv_bfloat16 *>(bk.param_lp), bk.n, tiles};
+                p.g[nb] = bk.grads[worker];
+                p.snap[nb] = static_cast<const float *>(snapshots[i]);
+                tiles += (bk.n + ki.tile - 1) / ki.tile;
+                ++nb;
+            }
+            if (nb == 0) break;
+            p.eta = float(eta_k); p.wd = weight_decay;
+            p.nb = nb;
+            p.tiles = tiles;
+            const int grid = tiles < (unsigned long long)shape.grid ? int(tiles) : shape.grid;
+            rc = launch(ctx, ki, grid, &p, s);
+            if (rc != OMNI_OK) return rc;
+        }
+        if (write_back)   // the register family pulls with plain device copies
+            for (int j = 0; j < n_buckets; ++j)
+                if (buckets[j].n)
+                    OMNI_CUDA(ctx, cudaMemcpyAsync(snapshots[j], buckets[j].param, buckets[j].n * sizeof(float),
+                                                   cudaMemcpyDeviceToDevice, s));
     }
     ctx->tally.arrivals += 1;
     ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
     if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
     return OMNI_OK;
+}
+
+int omni_asp_push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                            int32_t worker, int32_t b_used, int32_t tau, const void *const *snapshots, float lr,
+                            float weight_decay, void *stream)
+{
+    return push_overwrite(ctx, buckets, n_buckets, grad_dtype, worker, b_used, tau,
+                          const_cast<void *const *>(snapshots), false, lr, weight_decay, stream);
+}
+
+int omni_asp_push_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                       int32_t worker, int32_t b_used, int32_t tau, void *const *snapshots, float lr,
+                       float weight_decay, void *stream)
+{
+    return push_overwrite(ctx, buckets, n_buckets, grad_dtype, worker, b_used, tau, snapshots, true, lr, weight_decay,
+                          stream);
 }
 
 // ---- device-resident controller ----------------------------------------------------------------

@@ -11,6 +11,11 @@
 // (K = 1: a single arrival), lam[k] carries eta_k, and each element goes through the K
 // per-arrival updates in order instead of one weighted sum and one update; no norm is produced.
 //
+// OVW = true (with SEQ, one stream, no momentum) is the push with overwrite of Algorithm 2 on the
+// same ring: the "theta" slot of a stage is filled from the worker's snapshot (p.src) instead of
+// the server copy, the result replaces the server copy, and where p.copy is set it is also
+// written there (the worker's pull that follows its push, fused into the same pass).
+//
 // Every wait on an mbarrier is bounded: when the limit is hit the thread records it in the
 // workspace status word and leaves the kernel; the host reports OMNI_ERR_TIMEOUT.
 // Bulk copies need 16-byte aligned addresses and sizes, which the library's alignment contract
@@ -122,7 +127,7 @@ template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int 
     return tma_ring_bytes(tma_shape<G>(K), K, int(sizeof(G)));
 }
 
-template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false, bool DEVLAM = false>
+template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false, bool DEVLAM = false, bool OVW = false>
 __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_constant__ BspParams p)
 {
     constexpr int THREADS = (NCW + 1) * 32;
@@ -182,7 +187,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                 mbar_expect_tx(&full[s], K * GB + FB + (with_v ? FB : 0u));
 #pragma unroll
                 for (int k = 0; k < K; ++k) bulk_load(st + k * GB, static_cast<const G *>(p.g[bi][k]) + base, GB, &full[s], pol_stream);
-                bulk_load(st + K * GB, bd.theta + base, FB, &full[s], pol_keep);
+                if constexpr (OVW) bulk_load(st + K * GB, p.src[bi] + base, FB, &full[s], pol_stream);
+                else bulk_load(st + K * GB, bd.theta + base, FB, &full[s], pol_keep);
                 if (with_v) bulk_load(st + K * GB + FB, bd.v + base, FB, &full[s], pol_keep);
             }
             // Leave no copy in flight when this CTA gives its shared memory back: the stages armed
@@ -215,6 +221,9 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
             const BucketDesc bd = p.bk[bi];
             const unsigned long long base = (tile - bd.tile0) * TILE;
             const bool has_v = bd.v != nullptr, has_lp = bd.lp != nullptr;
+            const float *tsrc = bd.theta;      // where the ragged path reads the "theta" operand
+            float *cpy = nullptr;              // second destination of the result (OVW: the snapshot)
+            if constexpr (OVW) { tsrc = p.src[bi]; cpy = p.copy[bi]; }
             if (!mbar_wait(&full[s], unsigned((i / STAGES) & 1))) {
                 atomicExch(&p.ws->status, kStatusTimeout);
                 break;
@@ -287,6 +296,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                         if (has_v) store_floats_policy<E>(bd.v + off, vv, pol_keep);
                     }
                     if (has_lp) store_lp<E / 2>(bd.lp + off, th);
+                    if constexpr (OVW) { if (cpy) store_floats<4, E / 4>(cpy + off, th); }
                 }
             } else {
                 // ragged tile from global memory: whole 16-byte vectors, then single elements
@@ -296,7 +306,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                         Raw<4> raw[K];
 #pragma unroll
                         for (int k = 0; k < K; ++k) raw[k] = ld_ro<4>(static_cast<const G *>(p.g[bi][k]) + off);
-                        load_floats<4, V / 4>(bd.theta + off, th);
+                        load_floats<4, V / 4>(tsrc + off, th);
                         if (with_v) load_floats<4, V / 4>(bd.v + off, vv);
                         if constexpr (SEQ) {
 #pragma unroll
@@ -329,10 +339,11 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                         store_floats<4, V / 4>(bd.theta + off, th);
                         if (has_v) store_floats<4, V / 4>(bd.v + off, vv);
                         if (has_lp) store_lp<V / 2>(bd.lp + off, th);
+                        if constexpr (OVW) { if (cpy) store_floats<4, V / 4>(cpy + off, th); }
                     } else {
                         for (unsigned long long j = off; j < bd.n; ++j) {
                             float vj = with_v ? __ldcs(bd.v + j) : 0.0f;
-                            float t = __ldcs(bd.theta + j);
+                            float t = __ldcs(tsrc + j);
                             if constexpr (SEQ) {
 #pragma unroll
                                 for (int k = 0; k < K; ++k)
@@ -348,6 +359,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                             bd.theta[j] = t;
                             if (has_v) bd.v[j] = vj;
                             if (has_lp) bd.lp[j] = __float2bfloat16_rn(t);
+                            if constexpr (OVW) { if (cpy) cpy[j] = t; }
                         }
                     }
                 }

@@ -350,12 +350,13 @@ def test_asp_batched_apply_equals_successive_arrivals(kind, mu, wd):
     assert L.omni_apply_asp_batch(h, bs.array, 1, bs.dtype, 2, i32(0, 1), i32(8, 8), i32(0, -1), 0.1, mu, wd, None) == B.ERR_BAD_TAU
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("kind", ["f32", "bf16"])
-def test_asp_pull_and_push_with_overwrite(kind):
+def test_asp_pull_and_push_with_overwrite(kind, fused):
     """Algorithm 2 literally on a shrunk model: workers pull snapshots at different times and
     push with overwrite; the event stream (with controller feedback) runs on both sides; the
     server copy matches the oracle bit for bit after every event, and differs from what applying
-    the same gradients would give."""
+    the same gradients would give.  fused: the push and the worker's next pull in one call."""
     base = W.config("resnet50_asp")
     cfg = W.scaled(W.Config(**{**base.__dict__, "grad_dtype": kind}), 500)
     buf = W.make_buffers(cfg, DEV)
@@ -384,8 +385,11 @@ def test_asp_pull_and_push_with_overwrite(kind):
     for i in range(300):
         k = W.pick_worker(u[i], [T[j] / b[j] for j in range(K)])
         tau = i - last[k]
-        o.asp_push_overwrite(bs, k, b[k], tau, [snaps[k][s] for s in sl], cfg.lr, 1e-4)
-        o.asp_pull(bs, [snaps[k][s] for s in sl])                             # next iteration starts with a pull
+        if fused:
+            o.asp_push_pull(bs, k, b[k], tau, [snaps[k][s] for s in sl], cfg.lr, 1e-4)
+        else:
+            o.asp_push_overwrite(bs, k, b[k], tau, [snaps[k][s] for s in sl], cfg.lr, 1e-4)
+            o.asp_pull(bs, [snaps[k][s] for s in sl])                         # next iteration starts with a pull
         for s in sl:                                                          # the oracle walks the same buckets
             O.asp_push_overwrite_f32(g_np[k][s], b[k], cfg.global_batch, th_o[s], snaps_o[k][s], cfg.lr, 1e-4, theta_lp=lp_o[s])
         snaps_o[k][:] = th_o
@@ -398,7 +402,9 @@ def test_asp_pull_and_push_with_overwrite(kind):
         if i % 50 == 0 or i == 299:
             assert np.array_equal(to_np(buf.theta), th_o), i
     assert np.array_equal(to_np(lp), lp_o)
-    assert np.array_equal(to_np(snaps[3]), snaps_o[3])
+    for k in range(K):
+        for s_ in sl:
+            assert np.array_equal(to_np(snaps[k][s_]), snaps_o[k][s_]), k
     st = o.stats()
     assert st.arrivals == 300 and st.tau_hist == tally.hist.tolist() and st.tau_max == tally.tau_max
     real = np.concatenate([np.arange(a, a + n) for _, a, n in lay.tensor_slices()])
