@@ -177,3 +177,19 @@ def test_argument_validation_happens_before_any_cuda_call():
     assert o.kernel_launches == 0
     s = o.stats()
     assert s.steps == 0 and s.arrivals == 0 and sum(s.tau_hist) == 0
+
+
+def test_the_abi_is_usable_from_plain_c(tmp_path):
+    """include/omni.h compiles as C99 with warnings as errors, and a C program linked against the
+    library runs the host controller (no GPU involved)."""
+    import subprocess
+
+    lib = B._build.build()
+    exe = tmp_path / "controller_from_c"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", str(ROOT / "include"),
+                    str(ROOT / "tests" / "c_abi" / "controller_from_c.c"), "-o", str(exe),
+                    str(lib), f"-Wl,-rpath,{lib.parent}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.splitlines()
+    assert out[:4] == ["2 6 19 37", "6 9 17 32", "4 8 16 36", "4 8 16 36"]
+    assert out[4].startswith(f"{B.ERR_NULL} ")
+    assert out[5] == "0+384 384+320 704+296"
