@@ -216,3 +216,64 @@ def test_whole_steps_replayed_from_a_cuda_graph():
     assert np.array_equal(to_np(theta), th_o) and np.array_equal(to_np(v), v_o)
     assert o.ctl_from_device() == [int(x) for x in ref.batches]
     assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+
+
+def test_mixed_call_sequence_on_one_context_and_stream():
+    """Two hundred calls of every kind back to back on one stream and one set of buffers --
+    synchronous steps with host and with device-resident weights, single and batched
+    asynchronous arrivals, push + pull in one pass, the allocation-free step -- with no
+    synchronisation in between: the kernels order themselves (dependent launches, alternating
+    sweep directions, shared workspace).  State after every twentieth call and at the end equals
+    the oracle's, bit for bit."""
+    K, n, B_ = 5, 3 * 8192 + 1031, 160
+    gen = torch.Generator(device=DEV).manual_seed(4242)
+    theta = torch.empty(n, device=DEV).normal_(0, 0.05, generator=gen)
+    v = torch.zeros(n, device=DEV)
+    snap = theta.clone()
+    grads = [torch.empty(n, device=DEV).normal_(0, 1e-3, generator=gen) for _ in range(K)]
+    o = B.Omni(K, B_, 4, 96, 0.10)
+    ref = O.Controller(K, B_, 4, 96, 0.10)
+    bs = B.BucketSet([theta], [grads], [v])
+    th_o, v_o, sn_o, g_np = to_np(theta), to_np(v), to_np(snap), [to_np(g) for g in grads]
+    rng = np.random.default_rng(17)
+    measured = torch.empty(K, dtype=torch.float64, device=DEV)
+    o.ctl_to_device()
+    lr, mu, wd = 0.05, 0.9, 1e-4
+    for i in range(200):
+        kind = int(rng.integers(0, 6))
+        if kind == 0:
+            b = [int(x) for x in ref.batches]
+            o.aggregate_bsp(bs, b, lr, mu, wd)
+            O.bsp_step_f32(g_np, b, th_o, v_o, lr, mu, wd)
+        elif kind == 1:
+            T = 8.0 ** rng.random(K)
+            measured.copy_(torch.from_numpy(T))
+            o.rebatch_device(measured)
+            ref.rebatch(T)
+            o.aggregate_bsp_device_batches(bs, lr, mu, wd)
+            O.bsp_step_f32(g_np, ref.batches, th_o, v_o, lr, mu, wd)
+        elif kind == 2:
+            k, bu = int(rng.integers(0, K)), int(rng.integers(4, 97))
+            o.apply_asp(bs, k, bu, 0, lr, mu, wd)
+            O.asp_apply_f32(g_np[k], bu, B_, th_o, v_o, lr, mu, wd)
+        elif kind == 3:
+            ks = [int(x) for x in rng.integers(0, K, 3)]
+            bus = [int(x) for x in rng.integers(4, 97, 3)]
+            o.apply_asp_batch(bs, ks, bus, [0, 1, 2], lr, mu, wd)
+            for k, bu in zip(ks, bus):
+                O.asp_apply_f32(g_np[k], bu, B_, th_o, v_o, lr, mu, wd)
+        elif kind == 4:
+            k, bu = int(rng.integers(0, K)), int(rng.integers(4, 97))
+            o.asp_push_pull(bs, k, bu, 0, [snap], lr, wd)
+            O.asp_push_overwrite_f32(g_np[k], bu, B_, th_o, sn_o, lr, wd)
+            sn_o[:] = th_o
+        else:
+            b = [int(x) for x in ref.batches]
+            B.aggregate_bsp_noalloc(bs, b, lr, mu, wd)
+            O.bsp_step_f32(g_np, b, th_o, v_o, lr, mu, wd)
+        if i % 20 == 19:
+            assert np.array_equal(to_np(theta), th_o), i
+            assert np.array_equal(to_np(v), v_o), i
+    assert np.array_equal(to_np(snap), sn_o)
+    assert o.ctl_from_device() == [int(x) for x in ref.batches]
+    o.stats()                                            # no bounded wait ran out
