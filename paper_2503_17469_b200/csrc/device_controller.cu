@@ -46,24 +46,37 @@ __global__ void __launch_bounds__(32) rebatch_kernel(DeviceCtl *c, const CtlCons
     const int k = threadIdx.x;
     const bool on = k < cc.K;
 
+    // Launched with programmatic stream serialization: the step that follows may take its SMs and
+    // set up while this warp works, and nothing is read here before the previous launch (a step
+    // that read the weights, or whatever produced the measurements) has finished.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     // a measurement that is not a positive finite number fails the call; nothing changes
+    // all of this lane's state is fetched at once (one memory latency instead of three in a row)
     const double m = on ? measured[k] : 1.0;
+    const int32_t b = on ? c->batch[k] : 1;
+    const int32_t seen = on ? c->seen[k] : 0;
+    const double prev = on ? c->time[k] : 0.0;
     if (__any_sync(kFull, on && !(isfinite(m) && m > 0.0))) {
         if (k == 0) atomicCAS(&c->status, 0, int(OMNI_ERR_BAD_MEASUREMENT));
         return;
     }
-    const int32_t b = on ? c->batch[k] : 1;
     const double bd = double(b);
     const double lo = double(cc.b_min), hi = double(cc.b_max);
 
     // Eq. 6a read backwards (t = b / T), then the EWMA of the compute time; the first sample seeds it
     const double t = (cc.flags & OMNI_INPUT_IS_TIME) ? m : __ddiv_rn(bd, m);
     double s = t;
-    if (on && c->seen[k]) s = __dadd_rn(__dmul_rn(cc.alpha, t), __dmul_rn(__dsub_rn(1.0, cc.alpha), c->time[k]));
+    if (seen) s = __dadd_rn(__dmul_rn(cc.alpha, t), __dmul_rn(__dsub_rn(1.0, cc.alpha), prev));
 
     // mean compute time, summed in ascending k by every lane
     double total = 0.0;
-    for (int j = 0; j < cc.K; ++j) total = __dadd_rn(total, __shfl_sync(kFull, s, j));
+#pragma unroll
+    for (int j = 0; j < OMNI_MAX_K; ++j) {
+        const double sj = __shfl_sync(kFull, s, j);
+        if (j < cc.K) total = __dadd_rn(total, sj);
+    }
     const double tbar = __ddiv_rn(total, double(cc.K));
 
     // getBsz: Eq. 6b, dead-band (Eq. 7), bounds, one rounding to an integer (half up)
@@ -117,22 +130,16 @@ __global__ void __launch_bounds__(32) rebatch_kernel(DeviceCtl *c, const CtlCons
 
     // commit, then the weights of Eq. 4b for the step that follows
     const long long sum_b = warp_sum(on ? n : 0);
-    float lam = 0.0f;
     if (on) {
         c->batch[k] = n;
         c->time[k] = s;
         c->seen[k] = 1;
         if (new_b) new_b[k] = n;
-        lam = __double2float_rn((cc.flags & OMNI_UNSCALED_MEAN) ? __ddiv_rn(1.0, double(cc.K))
+        const float lam = __double2float_rn((cc.flags & OMNI_UNSCALED_MEAN) ? __ddiv_rn(1.0, double(cc.K))
                                                                   : __ddiv_rn(double(n), double(sum_b)));
         c->lam[k] = lam;
     }
-    double wsum = 0.0;
-    for (int j = 0; j < cc.K; ++j) wsum = __dadd_rn(wsum, double(__shfl_sync(kFull, lam, j)));
-    if (k == 0) {
-        c->weight_sum = wsum;
-        c->rebatches += 1u;
-    }
+    if (k == 0) c->rebatches += 1u;     // (the sum of the weights is taken on the host when the state is read back)
 }
 
 template <typename G, int K> KernelInfo devlam_info()
@@ -166,8 +173,16 @@ int launch_device_rebatch(DeviceCtl *ctl, const omni_config &cfg, const double *
                           void *stream)
 {
     const CtlConst cc{cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.mode, cfg.flags, cfg.deadband, cfg.ewma_alpha};
-    rebatch_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctl, cc, measured_dev, new_b_dev);
-    return int(cudaGetLastError());
+    cudaLaunchConfig_t cfgl = {};
+    cfgl.gridDim = dim3(1);
+    cfgl.blockDim = dim3(32);
+    cfgl.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfgl.attrs = attr;
+    cfgl.numAttrs = 1;
+    return int(cudaLaunchKernelEx(&cfgl, rebatch_kernel, ctl, cc, measured_dev, new_b_dev));
 }
 
 }  // namespace omni

@@ -17,7 +17,7 @@ struct DeviceCtl {
     int32_t batch[OMNI_MAX_K];   // b_k
     int32_t seen[OMNI_MAX_K];    // 0 until the worker's first measurement has seeded the EWMA
     float lam[OMNI_MAX_K];       // lambda_k = float(b_k / sum b)  (1/K with OMNI_UNSCALED_MEAN)
-    double weight_sum;           // sum of lam as doubles, ascending k
+    double weight_sum;           // sum of lam as doubles, ascending k (filled on the host side of a download)
     int32_t status;              // 0, or the omni_status of the first device re-batch that failed since the last read
     uint32_t rebatches;          // device re-batches that completed
 };

@@ -752,6 +752,8 @@ int omni_ctl_from_device(omni_ctx *ctx, void *stream)
     OMNI_CUDA(ctx, cudaMemcpyAsync(&st, ctx->dctl, sizeof st, cudaMemcpyDeviceToHost, s));
     OMNI_CUDA(ctx, cudaStreamSynchronize(s));
     ctx->ctl.import_state(st.batch, st.time, st.seen);
+    st.weight_sum = 0.0;
+    for (int k = 0; k < ctx->ctl.K(); ++k) st.weight_sum += double(st.lam[k]);
     ctx->tally.weight_sum = st.weight_sum;
     if (st.status != 0) {
         // a device re-batch refused its input since the last read: report it once and clear it
