@@ -320,7 +320,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="omni", choices=["omni", "reference"])
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--extras", default="all", choices=["all", "none", "asp"],
+    ap.add_argument("--extras", default="all", choices=["all", "none", "asp", "ksweep"],
                     help="which of the other configurations to time as well (not part of `value`)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -382,7 +382,10 @@ def main():
 
     extras = {}
     if rank == 0 and world == 1 and not args.no_extras and args.extras != "none":
-        extras = run_extras(torch, W, B, peak, job, only_asp=args.extras == "asp")
+        if args.extras == "ksweep":
+            extras = run_k_sweep(torch, B, peak)
+        else:
+            extras = run_extras(torch, W, B, peak, job, only_asp=args.extras == "asp")
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -418,6 +421,44 @@ def main():
         }
         print(json.dumps(line))
     ranks.close()
+
+
+def run_k_sweep(torch, B, peak, P=25_557_032, steps=200):
+    """The synchronous step on one flat bucket of P parameters for a range of worker counts and both
+    gradient types (fixed batches, momentum 0.9): algorithmic GB/s against the measured copy peak."""
+    out = {}
+    dev = torch.device("cuda", torch.cuda.current_device())
+    gen = torch.Generator(device=dev).manual_seed(0x0517)
+    theta = torch.empty(P, device=dev).normal_(0, 0.05, generator=gen)
+    v = torch.zeros(P, device=dev)
+    for kind, gdt, esz in (("f32", torch.float32, 4), ("bf16", torch.bfloat16, 2)):
+        grads = []
+        for K in (1, 2, 4, 8, 12, 16, 20, 24, 32):
+            while len(grads) < K:
+                grads.append(torch.empty(P, device=dev).normal_(0, 1e-3, generator=gen).to(gdt))
+            o = B.Omni(K, 32 * K, 4, 96, 0.10)
+            bs = B.BucketSet([theta], [grads[:K]], [v])
+            b = o.batches
+            for _ in range(5):
+                o.aggregate_bsp(bs, b, 0.1, 0.9)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                o.aggregate_bsp(bs, b, 0.1, 0.9)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / steps
+            bpp = esz * K + 16
+            gbs = bpp * P / (ms * 1e-3) / 1e9
+            grid, block = o.query_launch(K, B.BF16 if kind == "bf16" else B.F32)
+            out[f"{kind}_K{K}"] = {"ms_per_step": ms, "bytes_per_param": bpp, "achieved_gbs": gbs,
+                                   "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+                                   "params_per_s": P / (ms * 1e-3), "grid": grid, "block": block}
+            del o, bs
+        del grads
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_extras(torch, W, B, peak, headline_job, only_asp=False):
