@@ -600,3 +600,39 @@ def test_resnet50_asp_full_size_sampled():
         for k, bu, tau in events:
             O.asp_apply_f32(g_np[k], bu, cfg.global_batch, th_o, None, cfg.lr, 0.0, 0.0)
         assert np.array_equal(to_np(buf.theta[s:e]), th_o), (s, e)
+
+
+def test_bucket_longer_than_32_bit_indices():
+    """One bucket of 2^32 + 197,637 elements (bf16 gradient, no momentum buffer: 26 GB on the device):
+    element offsets do not fit 32 bits.  The oracle checks windows at the start, across 2^31 and
+    2^32, and the ragged tail; between the windows the gradient is zero and theta constant, so
+    samples there must equal the one value the oracle gives for such an element, and the squared
+    norm is the windows' alone."""
+    n = (1 << 32) + 3 * 65536 + 1029
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30):
+        pytest.skip("needs 40 GB of free device memory")
+    gen = _gen(2**20 + 3)
+    theta = torch.empty(n, device=DEV, dtype=torch.float32)
+    grad = torch.zeros(n, device=DEV, dtype=torch.bfloat16)
+    theta.fill_(0.25)
+    w = 1 << 16
+    windows = [0, (1 << 31) - w // 2, (1 << 32) - w // 2, n - w]
+    for a in windows:                                   # random values only where the oracle will look
+        theta[a:a + w].normal_(0, 0.05, generator=gen)
+        grad[a:a + w] = torch.empty(w, device=DEV).normal_(0, 1e-3, generator=gen).to(torch.bfloat16)
+    before = [(to_np(theta[a:a + w]), to_np(grad[a:a + w])) for a in windows]
+    o = B.Omni(1, 32, 1, 96, 0.1)
+    o.aggregate_bsp(B.BucketSet([theta], [[grad]]), [32], 0.1, 0.0, 1e-3)
+    sq_want = 0.0
+    for a, (th_o, g_o) in zip(windows, before):
+        sq_want += O.bsp_step_f32([g_o], [32], th_o, None, 0.1, 0.0, 1e-3)
+        assert np.array_equal(to_np(theta[a:a + w]), th_o), a
+    # everywhere else the gradient is zero and theta is one value: the oracle says what it becomes
+    flat = np.full(8, 0.25, np.float32)
+    O.bsp_step_f32([np.zeros(8, np.uint16)], [32], flat, None, 0.1, 0.0, 1e-3)
+    want_rest = flat[0]
+    for a in (w + 12345, (1 << 31) + (1 << 20), (1 << 32) - (1 << 20), (1 << 32) + w + 7):
+        got = to_np(theta[a:a + 4096])
+        assert (got == want_rest).all(), a
+    assert abs(o.stats().grad_sqnorm - sq_want) <= SQNORM_RTOL * sq_want
