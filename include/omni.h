@@ -114,6 +114,18 @@ int omni_get_batches(const omni_ctx *ctx, int32_t *b);
 /* Overwrite them.  BAD_BATCH if some b_k < 1 or, in BSP mode, sum != B. */
 int omni_set_batches(omni_ctx *ctx, const int32_t *b);
 
+/* Controller state for checkpoints (the paper notes that a batch re-adjustment goes through a
+ * checkpoint of the job, Sec. III-B): the batches, the smoothed compute times and which workers
+ * have one yet, as one flat record.  omni_ctl_export: *size (host, in/out) holds the capacity of
+ * `record` (host) and receives the record's size; record == NULL only queries the size.
+ * omni_ctl_import restores a record into a context created with the same K and global batch;
+ * batch sizes and times are validated and a failed import changes nothing.  Parameter buffers,
+ * momentum and the device copy of the controller are the caller's to save.
+ * Errors: NULL, TOO_LARGE (capacity below the record's size), BAD_CONFIG (not a record, or made
+ * for another K or global batch), BAD_BATCH, BAD_MEASUREMENT. */
+int omni_ctl_export(const omni_ctx *ctx, void *record, uint64_t *size);
+int omni_ctl_import(omni_ctx *ctx, const void *record, uint64_t size);
+
 /* Synchronous re-batch: getAvgComputeTime + getBsz for every worker (Algorithm 1) + Eq. 8.
  * measured[K] (host): throughput T_k in samples per time unit seen with the current b_k, or the
  * compute time t_k if OMNI_INPUT_IS_TIME.  Steps, all in IEEE double, sums in ascending k:

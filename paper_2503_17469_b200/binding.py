@@ -29,7 +29,7 @@ EXPORTS = (
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
     "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
     "omni_ctl_to_device", "omni_ctl_from_device", "omni_rebatch_device", "omni_aggregate_bsp_device_batches",
-    "omni_shard_range", "omni_asp_push_pull",
+    "omni_shard_range", "omni_asp_push_pull", "omni_ctl_export", "omni_ctl_import",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
     L.omni_rebatch_device.argtypes = [vp, vp, vp, vp]
     L.omni_aggregate_bsp_device_batches.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, f32, f32, f32, vp]
     L.omni_shard_range.argtypes = [C.c_uint64, i32, i32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    L.omni_ctl_export.argtypes = [vp, vp, C.POINTER(C.c_uint64)]
+    L.omni_ctl_import.argtypes = [vp, vp, C.c_uint64]
     L.omni_selftest_wait_expiry.argtypes = [vp, vp]
     L.omni_last_cuda_error.argtypes = [vp]
     L.omni_query_launch.argtypes = [vp, i32, i32, C.POINTER(i32), C.POINTER(i32)]
@@ -253,6 +255,17 @@ class Omni:
         nb = self._i32K()
         self._check(lib().omni_rebatch_static(self._h, self._f64K(*capacity), nb))
         return list(nb)
+
+    def export_state(self) -> bytes:
+        """The controller state (batches, smoothed times) as bytes, for a checkpoint."""
+        size = C.c_uint64(0)
+        self._check(lib().omni_ctl_export(self._h, None, C.byref(size)))
+        buf = C.create_string_buffer(size.value)
+        self._check(lib().omni_ctl_export(self._h, buf, C.byref(size)))
+        return buf.raw[:size.value]
+
+    def import_state(self, record: bytes) -> None:
+        self._check(lib().omni_ctl_import(self._h, record, len(record)))
 
     # ---- device path ------------------------------------------------------------------------
     @staticmethod

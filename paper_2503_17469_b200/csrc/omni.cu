@@ -371,6 +371,52 @@ int omni_set_batches(omni_ctx *ctx, const int32_t *b)
     return ctx->ctl.set_batches(b);
 }
 
+// Controller state as a flat record for checkpoints: what re-batching needs to continue where it
+// stopped (the paper's re-batching goes through a checkpoint of the training job).
+namespace {
+struct CtlRecord {
+    uint32_t magic, version;
+    int32_t K, global_batch;
+    int32_t batch[OMNI_MAX_K];
+    int32_t seen[OMNI_MAX_K];
+    double time[OMNI_MAX_K];
+};
+constexpr uint32_t kCtlMagic = 0x4c544d4fu;   // "OMTL"
+}  // namespace
+
+int omni_ctl_export(const omni_ctx *ctx, void *record, uint64_t *size)
+{
+    if (!ctx || !size) return OMNI_ERR_NULL;
+    const uint64_t have = *size;
+    *size = sizeof(CtlRecord);
+    if (!record) return OMNI_OK;                       // size query
+    if (have < sizeof(CtlRecord)) return OMNI_ERR_TOO_LARGE;
+    CtlRecord r{};
+    r.magic = kCtlMagic;
+    r.version = 1;
+    r.K = ctx->ctl.K();
+    r.global_batch = ctx->ctl.B();
+    ctx->ctl.export_state(r.batch, r.time, r.seen);
+    std::memcpy(record, &r, sizeof r);
+    return OMNI_OK;
+}
+
+int omni_ctl_import(omni_ctx *ctx, const void *record, uint64_t size)
+{
+    if (!ctx || !record) return OMNI_ERR_NULL;
+    if (size < sizeof(CtlRecord)) return OMNI_ERR_BAD_CONFIG;
+    CtlRecord r;
+    std::memcpy(&r, record, sizeof r);
+    if (r.magic != kCtlMagic || r.version != 1 || r.K != ctx->ctl.K() || r.global_batch != ctx->ctl.B())
+        return OMNI_ERR_BAD_CONFIG;
+    for (int k = 0; k < r.K; ++k)
+        if (r.seen[k] && !(std::isfinite(r.time[k]) && r.time[k] > 0.0)) return OMNI_ERR_BAD_MEASUREMENT;
+    const int rc = ctx->ctl.set_batches(r.batch);      // validates b_k >= 1 and, in BSP mode, the sum
+    if (rc != OMNI_OK) return rc;
+    ctx->ctl.import_state(r.batch, r.time, r.seen);
+    return OMNI_OK;
+}
+
 int omni_rebatch(omni_ctx *ctx, const double *measured, int32_t *new_b, int32_t *changed)
 {
     if (!ctx || !measured || !new_b) return OMNI_ERR_NULL;

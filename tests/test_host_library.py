@@ -193,3 +193,35 @@ def test_the_abi_is_usable_from_plain_c(tmp_path):
     assert out[:4] == ["2 6 19 37", "6 9 17 32", "4 8 16 36", "4 8 16 36"]
     assert out[4].startswith(f"{B.ERR_NULL} ")
     assert out[5] == "0+384 384+320 704+296"
+
+
+def test_controller_state_survives_a_checkpoint():
+    """Export after some re-batches with EWMA smoothing, import into a fresh context: both continue
+    with identical batches; records for another configuration or damaged records are refused and
+    leave the context as it was."""
+    mk = lambda K=4, Bt=128: B.Omni(K, Bt, 4, 96, 0.05, ewma_alpha=0.5)
+    a = mk()
+    rng = np.random.default_rng(3)
+    for _ in range(3):
+        a.rebatch(list(8.0 ** rng.random(4)))
+    rec = a.export_state()
+    b = mk()
+    b.import_state(rec)
+    assert b.batches == a.batches
+    for _ in range(5):
+        T = list(8.0 ** rng.random(4))
+        assert a.rebatch(T) == b.rebatch(T)           # the smoothed times came along
+    for bad_ctx in (mk(K=8, Bt=256), mk(Bt=160)):
+        with pytest.raises(B.OmniError) as e:
+            bad_ctx.import_state(rec)
+        assert e.value.status == B.ERR_BAD_CONFIG
+    c = mk()
+    before = c.batches
+    for damaged in (rec[:40], b"\0" * len(rec)):
+        with pytest.raises(B.OmniError):
+            c.import_state(damaged)
+    broken = bytearray(rec)
+    broken[16:20] = (0).to_bytes(4, "little", signed=True)      # batch[0] = 0
+    with pytest.raises(B.OmniError) as e:
+        c.import_state(bytes(broken))
+    assert e.value.status == B.ERR_BAD_BATCH and c.batches == before
