@@ -105,17 +105,26 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
     if (tile * int(sizeof(G)) < 4096 && 2 * (tile * 3 / 2) * per_elem <= 216 * 1024) tile = tile * 3 / 2;
     const int stage = tile * per_elem;
     int stages = (152 * 1024 + stage / 2) / stage;
+    // float K = 12, 13: three 56-60 KB stages (168-180 KB) lose 3 % to two (7.03 vs 7.22, 6.98 vs 7.23 TB/s)
+    if (sizeof(G) == 4 && tile == 1024 && stages * stage > 160 * 1024) stages = 2;
     if (stages < 2) stages = 2;
     if (stages > 8) stages = 8;
     return {tile, stages, 8};
 }
-// The asynchronous apply of M queued arrivals uses the same geometry with M streams, except the
-// single float arrival: with most of theta coming from L2 (see the alternating sweeps in
-// omni.cu) it is no longer DRAM-bound, and four stages with sixteen consumer warps gain 3 %
-// (8.20 vs 7.96 TB/s algorithmic).
+// The asynchronous apply of M queued arrivals uses the same geometry with M streams, except for
+// the shortest queues: with most of theta coming from L2 (see the alternating sweeps in omni.cu)
+// they are no longer DRAM-bound, and a deeper ring with sixteen consumer warps gains 2-6 %
+// (float M = 1: 8.20 vs 7.96 TB/s algorithmic; M = 2: 8.70 vs 8.24; M = 3: 8.55 vs 8.38;
+// bfloat16 M = 1: 8.73 vs 8.59; from M = 4 on nothing changed).
 template <typename G> __host__ __device__ constexpr TmaShape tma_seq_shape(int M)
 {
-    if (M == 1 && sizeof(G) == 4) return {4096, 4, 16};
+    if (sizeof(G) == 4) {
+        if (M == 1) return {4096, 4, 16};
+        if (M == 2) return {4096, 3, 16};
+        if (M == 3) return {2048, 4, 16};
+    } else if (M == 1) {
+        return {4096, 4, 16};
+    }
     return tma_shape<G>(M);
 }
 __host__ __device__ constexpr unsigned tma_ring_bytes(TmaShape s, int streams, int gsize)
