@@ -98,11 +98,27 @@ def test_asp_report_bit_exact_against_oracle():
         for ev in range(200):
             k = int(rng.integers(0, K))
             meas = float(T[k] * (1 + 0.1 * rng.uniform(-1, 1)))
-            a = lib.asp_report(k, cur[k], meas)
-            b = ora.asp_report(k, cur[k], meas)
+            # now and then a worker ran another batch than the one the server handed it
+            used = cur[k] if rng.uniform() < 0.8 else int(rng.integers(4, 97))
+            a = lib.asp_report(k, used, meas)
+            b = ora.asp_report(k, used, meas)
             assert a == b
             cur[k] = a
         assert lib.batches == ora.batches.tolist()
+
+
+def test_asp_report_hand_derived_sequences():
+    """The library's evalBsz on the hand-derived report sequences (a reported batch that differs
+    from the server's entry, smoothed times): same integers as derived by hand."""
+    import json
+
+    gold = json.loads((ROOT / "tests" / "golden" / "controller_cases.json").read_text())
+    for case in gold["report_cases"]:
+        flags = B.INPUT_IS_TIME if case["input"] == "time" else 0
+        o = B.Omni(case["K"], case["B"], case["b_min"], case["b_max"], case["deadband"], case["alpha"], B.ASP, flags)
+        for r in case["reports"]:
+            assert o.asp_report(r["worker"], r["b_used"], r["measured"]) == r["returns"], case["name"]
+            assert o.batches == r["map_after"], case["name"]
 
 
 def test_static_rebatch_matches_oracle():

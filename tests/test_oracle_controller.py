@@ -207,6 +207,19 @@ def test_asp_report_waits_for_all_workers_then_recomputes_all():
     assert c.batches.sum() != g["B"]
 
 
+@pytest.mark.parametrize("case", GOLD["report_cases"], ids=lambda c: c["name"].split()[0])
+def test_hand_derived_report_sequences(case):
+    """Algorithm 2 evalBsz by hand: the server stores the batch the worker RAN (which need not be
+    the entry it holds) and the smoothed compute time, then re-evaluates every entry."""
+    flags = O.FLAG_INPUT_IS_TIME if case["input"] == "time" else 0
+    c = O.Controller(case["K"], case["B"], case["b_min"], case["b_max"], case["deadband"], case["alpha"],
+                     O.MODE_ASP, flags)
+    assert c.batches.tolist() == case["b0"]
+    for r in case["reports"]:
+        assert c.asp_report(r["worker"], r["b_used"], r["measured"]) == r["returns"]
+        assert c.batches.tolist() == r["map_after"]
+
+
 def test_errors_leave_state_untouched():
     c = O.Controller(4, 64, 2, 48, 0.1)
     before = c.batches.copy()

@@ -40,6 +40,11 @@ MUTANTS = [
     ("bfloat16 rounds half up, not half to even", "u += 0x7fffu + lsb;", "u += 0x8000u;"),
     ("overwrite starts from the server copy", "theta[j] = snapshot[j] - eta_k * d;", "theta[j] = theta[j] - eta_k * d;"),
     ("static split ignores the capacities", "double x = capacity[k] / csum * (double)c->B;", "double x = (double)c->B / (double)c->K;"),
+    ("asynchronous report keeps the server's entry instead of the batch the worker ran", "c->b[worker] = b_used;\n    smooth(c, worker,", "smooth(c, worker,"),
+    ("asynchronous report skips the smoothing", "smooth(c, worker, measured_time(c, b_used, measured));",
+     "c->s[worker] = measured_time(c, b_used, measured); c->seen[worker] = 1;"),
+    ("asynchronous report takes the time from the server's entry", "c->b[worker] = b_used;\n    smooth(c, worker, measured_time(c, b_used, measured));",
+     "smooth(c, worker, measured_time(c, c->b[worker], measured));\n    c->b[worker] = b_used;"),
     ("asynchronous report re-batches before everyone reported", "if (!all) { *new_b = b_used; return ORACLE_OK; }", "if (!all && worker < 0) { *new_b = b_used; return ORACLE_OK; }"),
 ]
 
