@@ -43,7 +43,8 @@ enum { ORACLE_MODE_BSP = 0, ORACLE_MODE_ASP = 1 };
 enum {
     ORACLE_FLAG_UNSCALED_MEAN = 1u,   /* ablation: lambda_k = 1/K (Table "weighted aggregation") */
     ORACLE_FLAG_ASP_NO_LR_SCALE = 2u, /* ablation: eta_k = eta (Table "LR scaling in ASP")       */
-    ORACLE_FLAG_INPUT_IS_TIME = 4u    /* measurements are compute times, not throughputs         */
+    ORACLE_FLAG_INPUT_IS_TIME = 4u,   /* measurements are compute times, not throughputs         */
+    ORACLE_FLAG_CONSERVE_MULTIPLICATIVE = 8u /* other reading of the sentence after Eq. 8, see oracle_rebatch */
 };
 enum {
     ORACLE_OK = 0,
@@ -119,12 +120,11 @@ static void smooth(oracle_ctl *c, int k, double x)
     else c->s[k] = c->alpha * x + (1.0 - c->alpha) * c->s[k];
 }
 
-/* getBsz of Alg. 1 for one worker, followed by the one rounding step to an integer.
+/* getBsz of Alg. 1 for one worker, real-valued:
  *   T  = b / t                                   (Eq. 6a)
  *   b* = b - T (t - tbar)                        (Eq. 6b)
- *   if |(b* - b) / b*| >= deadband: clamp b* to [b_min, b_max], else keep b     (Eq. 7, bounds)
- * reading: integer batch = floor(x + 1/2), clamped again so that rounding cannot leave the bounds. */
-static int32_t get_bsz(const oracle_ctl *c, int32_t b, double t, double tbar, double *bstar_out)
+ *   if |(b* - b) / b*| >= deadband: clamp b* to [b_min, b_max], else keep b     (Eq. 7, bounds) */
+static double get_bsz_real(const oracle_ctl *c, int32_t b, double t, double tbar, double *bstar_out)
 {
     double T = (double)b / t;
     double err = t - tbar;
@@ -138,10 +138,23 @@ static int32_t get_bsz(const oracle_ctl *c, int32_t b, double t, double tbar, do
     } else {
         cand = (double)b;
     }
+    return cand;
+}
+
+/* The one rounding step to an integer.
+ * reading: integer batch = floor(x + 1/2), clamped again so that rounding cannot leave the bounds. */
+static int32_t to_integer_batch(const oracle_ctl *c, double cand)
+{
     double r = floor(cand + 0.5);
     if (r < (double)c->b_min) r = (double)c->b_min;
     if (r > (double)c->b_max) r = (double)c->b_max;
     return (int32_t)r;
+}
+
+/* getBsz followed by the rounding step */
+static int32_t get_bsz(const oracle_ctl *c, int32_t b, double t, double tbar, double *bstar_out)
+{
+    return to_integer_batch(c, get_bsz_real(c, b, t, tbar, bstar_out));
 }
 
 /* Eq. 8: keep sum(b) = B by taking Delta B / K off every worker.
@@ -185,10 +198,20 @@ static int conserve_global_batch(const oracle_ctl *c, int32_t *n)
 /* One synchronous re-batch: getAvgComputeTime + getBsz for every worker + Eq. 8 (Alg. 1).
  * measured[k]: throughput of worker k in samples per time unit (or its compute time when the
  * INPUT_IS_TIME flag is set) observed while it ran batch b[k].
- * bstar_out (nullable) receives the real-valued b* of Eq. 6b, changed (nullable) 0/1 flags.
- * A failed call leaves the state untouched. */
+ * bstar_out (nullable) receives the real-valued b* of Eq. 6b, changed (nullable) 0/1 flags,
+ * scaled_out (nullable) the real-valued batches after the multiplicative renormalisation below
+ * (the getBsz values themselves without the flag).
+ * A failed call leaves the state untouched.
+ *
+ * The sentence after Eq. 8 (Sec. III-B, "Control Stability") says the adjusted batches are
+ * reduced "proportionately", while Eq. 8 itself subtracts the same Delta B / K from every worker.
+ * reading (default): the equation.  reading (CONSERVE_MULTIPLICATIVE, synchronous mode only): the
+ * real-valued getBsz results c_k of all workers are renormalised, c_k <- c_k * B / sum_i c_i,
+ * before the rounding step; whatever rounding and the bounds then leave of the gap to B is closed
+ * by the unit steps of the default reading.  From equal batches without dead-band and bounds this
+ * lands on B * T_k / sum(T) in one step, i.e. Eq. 4a with the throughputs as capacities. */
 int oracle_rebatch(oracle_ctl *c, const double *measured, int32_t *new_b, int32_t *changed,
-                   double *bstar_out)
+                   double *bstar_out, double *scaled_out)
 {
     oracle_ctl w = *c;
     int32_t n[ORACLE_MAX_K];
@@ -199,8 +222,23 @@ int oracle_rebatch(oracle_ctl *c, const double *measured, int32_t *new_b, int32_
     double tsum = 0.0;
     for (int k = 0; k < w.K; ++k) tsum += w.s[k];
     double tbar = tsum / (double)w.K;
-    for (int k = 0; k < w.K; ++k)
-        n[k] = get_bsz(&w, w.b[k], w.s[k], tbar, bstar_out ? &bstar_out[k] : NULL);
+    if (w.mode == ORACLE_MODE_BSP && (w.flags & ORACLE_FLAG_CONSERVE_MULTIPLICATIVE)) {
+        double cand[ORACLE_MAX_K], csum = 0.0;
+        for (int k = 0; k < w.K; ++k)
+            cand[k] = get_bsz_real(&w, w.b[k], w.s[k], tbar, bstar_out ? &bstar_out[k] : NULL);
+        for (int k = 0; k < w.K; ++k) csum += cand[k];
+        for (int k = 0; k < w.K; ++k) {
+            double scaled = cand[k] * (double)w.B / csum;
+            if (scaled_out) scaled_out[k] = scaled;
+            n[k] = to_integer_batch(&w, scaled);
+        }
+    } else {
+        for (int k = 0; k < w.K; ++k) {
+            double cand = get_bsz_real(&w, w.b[k], w.s[k], tbar, bstar_out ? &bstar_out[k] : NULL);
+            if (scaled_out) scaled_out[k] = cand;
+            n[k] = to_integer_batch(&w, cand);
+        }
+    }
     if (w.mode == ORACLE_MODE_BSP) {
         int rc = conserve_global_batch(&w, n);
         if (rc != ORACLE_OK) return rc;

@@ -21,7 +21,7 @@ _LIB = _HERE / "libomni_oracle.so"
 
 MAX_K = 32
 MODE_BSP, MODE_ASP = 0, 1
-FLAG_UNSCALED_MEAN, FLAG_ASP_NO_LR_SCALE, FLAG_INPUT_IS_TIME = 1, 2, 4
+FLAG_UNSCALED_MEAN, FLAG_ASP_NO_LR_SCALE, FLAG_INPUT_IS_TIME, FLAG_CONSERVE_MULTIPLICATIVE = 1, 2, 4, 8
 OK, ERR_ARG, ERR_INFEASIBLE, ERR_MEASUREMENT = 0, -1, -2, -3
 
 
@@ -53,7 +53,7 @@ def lib() -> C.CDLL:
         L.oracle_ctl_set_batches.argtypes = [vp, vp]
         L.oracle_ctl_get_batches.argtypes = [vp, vp]
         L.oracle_ctl_get_batches.restype = None
-        L.oracle_rebatch.argtypes = [vp, vp, vp, vp, vp]
+        L.oracle_rebatch.argtypes = [vp, vp, vp, vp, vp, vp]
         L.oracle_asp_report.argtypes = [vp, i32, i32, f64, vp]
         L.oracle_rebatch_static.argtypes = [vp, vp, vp]
         L.oracle_bsp_weights.argtypes = [i32, vp, u32, vp, vp]
@@ -135,16 +135,23 @@ class Controller:
         if rc != OK:
             raise OracleError(rc)
 
-    def rebatch(self, measured, want_bstar=False):
+    def rebatch(self, measured, want_bstar=False, want_scaled=False):
+        """(new batches, changed flags[, b* of Eq. 6b][, real-valued batches before rounding])."""
         m = np.ascontiguousarray(measured, np.float64)
         assert m.shape == (self.K,)
         nb = np.zeros(self.K, np.int32)
         ch = np.zeros(self.K, np.int32)
         bs = np.zeros(self.K, np.float64)
-        rc = lib().oracle_rebatch(self._buf, _ptr(m), _ptr(nb), _ptr(ch), _ptr(bs))
+        sc = np.zeros(self.K, np.float64)
+        rc = lib().oracle_rebatch(self._buf, _ptr(m), _ptr(nb), _ptr(ch), _ptr(bs), _ptr(sc))
         if rc != OK:
             raise OracleError(rc)
-        return (nb, ch, bs) if want_bstar else (nb, ch)
+        out = (nb, ch)
+        if want_bstar:
+            out += (bs,)
+        if want_scaled:
+            out += (sc,)
+        return out
 
     def rebatch_static(self, capacity) -> np.ndarray:
         c = np.ascontiguousarray(capacity, np.float64)

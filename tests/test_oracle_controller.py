@@ -220,6 +220,63 @@ def test_hand_derived_report_sequences(case):
         assert c.batches.tolist() == r["map_after"]
 
 
+@pytest.mark.parametrize("case", GOLD["multiplicative_cases"], ids=lambda c: c["name"].split()[0])
+def test_hand_derived_traces_multiplicative_conservation(case):
+    c = O.Controller(case["K"], case["B"], case["b_min"], case["b_max"], case["deadband"], 1.0, O.MODE_BSP,
+                     O.FLAG_CONSERVE_MULTIPLICATIVE)
+    assert c.batches.tolist() == case["b0"]
+    for want in case["expect"]:
+        assert c.rebatch(case["throughput"])[0].tolist() == want
+
+
+def test_multiplicative_conservation_lands_on_the_proportional_split_in_one_step():
+    """From equal batches, without dead-band and with wide bounds, the renormalised real-valued
+    batches are B * T_k / sum(T): Eq. 4a with the throughputs as capacities."""
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        K = int(rng.integers(2, 33))
+        T = rng.uniform(0.5, 20.0, K)
+        Bg = 32 * K
+        c = O.Controller(K, Bg, 1, 10**6, 0.0, 1.0, O.MODE_BSP, O.FLAG_CONSERVE_MULTIPLICATIVE)
+        nb, _, scaled = c.rebatch(T, want_scaled=True)
+        np.testing.assert_allclose(scaled, Bg * T / T.sum(), rtol=1e-12)
+        assert nb.sum() == Bg
+        # and the integers are the static split's, whenever no share sits within rounding noise of a half
+        frac = (Bg * T / T.sum()) % 1.0
+        if np.all(np.abs(frac - 0.5) > 1e-9):
+            s = O.Controller(K, Bg, 1, 10**6, 0.0, 1.0, O.MODE_BSP)
+            assert nb.tolist() == s.rebatch_static(T).tolist()
+
+
+def test_multiplicative_conservation_keeps_sum_and_bounds_exhaustively():
+    """Every initial split of small global batches over 2-3 workers, a grid of throughputs: after
+    the re-batch the sum is B and every batch is within the bounds; the asynchronous mode ignores
+    the flag (no global-batch rule there)."""
+    grid = [0.5, 1.0, 2.0, 3.5, 8.0]
+    for K in (2, 3):
+        for Bg in range(K * 2, 13):
+            b_min, b_max = 2, Bg - 2 * (K - 1)
+            for b0 in itertools.product(range(b_min, b_max + 1), repeat=K):
+                if sum(b0) != Bg:
+                    continue
+                for T in itertools.product(grid, repeat=K):
+                    for db in (0.0, 0.1):
+                        c = O.Controller(K, Bg, b_min, b_max, db, 1.0, O.MODE_BSP, O.FLAG_CONSERVE_MULTIPLICATIVE)
+                        c.set_batches(b0)
+                        nb, _ = c.rebatch(T)
+                        assert nb.sum() == Bg and nb.min() >= b_min and nb.max() <= b_max, (b0, T, db)
+    a = O.Controller(4, 128, 4, 96, 0.1, 1.0, O.MODE_ASP, O.FLAG_CONSERVE_MULTIPLICATIVE)
+    b = O.Controller(4, 128, 4, 96, 0.1, 1.0, O.MODE_ASP)
+    assert a.rebatch([4, 4, 4, 28])[0].tolist() == b.rebatch([4, 4, 4, 28])[0].tolist() == [25, 25, 25, 96]
+
+
+def test_equal_times_are_a_fixed_point_under_both_conservation_readings():
+    for flags in (0, O.FLAG_CONSERVE_MULTIPLICATIVE):
+        c = O.Controller(4, 64, 2, 48, 0.0, 1.0, O.MODE_BSP, flags)
+        c.set_batches([4, 8, 16, 36])
+        assert c.rebatch([1, 2, 4, 9])[0].tolist() == [4, 8, 16, 36]
+
+
 def test_errors_leave_state_untouched():
     c = O.Controller(4, 64, 2, 48, 0.1)
     before = c.batches.copy()

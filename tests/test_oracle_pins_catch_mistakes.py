@@ -45,6 +45,9 @@ MUTANTS = [
      "c->s[worker] = measured_time(c, b_used, measured); c->seen[worker] = 1;"),
     ("asynchronous report takes the time from the server's entry", "c->b[worker] = b_used;\n    smooth(c, worker, measured_time(c, b_used, measured));",
      "smooth(c, worker, measured_time(c, c->b[worker], measured));\n    c->b[worker] = b_used;"),
+    ("multiplicative conservation divides by the global batch, not by the sum of the proposals", "double scaled = cand[k] * (double)w.B / csum;", "double scaled = cand[k] * (double)w.B / (double)w.B;"),
+    ("multiplicative conservation scales the wrong way round", "double scaled = cand[k] * (double)w.B / csum;", "double scaled = cand[k] * csum / (double)w.B;"),
+    ("multiplicative conservation sums the old batches", "for (int k = 0; k < w.K; ++k) csum += cand[k];", "for (int k = 0; k < w.K; ++k) csum += (double)w.b[k];"),
     ("asynchronous report re-batches before everyone reported", "if (!all) { *new_b = b_used; return ORACLE_OK; }", "if (!all && worker < 0) { *new_b = b_used; return ORACLE_OK; }"),
 ]
 
