@@ -49,7 +49,8 @@ typedef enum {
     OMNI_ERR_CUDA = -9,            /* a CUDA call failed; see omni_last_cuda_error */
     OMNI_ERR_TIMEOUT = -10,        /* a bounded device-side wait ran out */
     OMNI_ERR_BAD_CONFIG = -11,     /* invalid omni_config field or call argument */
-    OMNI_ERR_TOO_LARGE = -12       /* size beyond a stated maximum */
+    OMNI_ERR_TOO_LARGE = -12,      /* size beyond a stated maximum */
+    OMNI_ERR_NO_MEMORY = -13       /* a host allocation failed */
 } omni_status;
 
 typedef enum { OMNI_BSP = 0, OMNI_ASP = 1 } omni_mode;
@@ -67,7 +68,16 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
  * touched last still in cache, and are launched with programmatic stream serialization (they
  * wait for the previous launch themselves, after their set-up).  The two flags force
  * one family; results are the same bit for bit.  A bounded wait of the ring that runs out
- * surfaces as OMNI_ERR_TIMEOUT from omni_get_stats. */
+ * surfaces as OMNI_ERR_TIMEOUT from omni_get_stats.
+ * Contract for the caller's own kernels on the same stream: the ring kernels (and the device
+ * re-batch kernel) signal "dependents may launch" (griddepcontrol.launch_dependents) as soon as
+ * their set-up is done, long before their last store.  A kernel enqueued after a library call
+ * in the ordinary way is not affected: the stream still runs it after the library's kernel has
+ * finished.  A kernel that the caller launches WITH the programmatic-stream-serialization
+ * attribute, however, may start while the library's kernel is still writing: it must execute
+ * griddepcontrol.wait (cudaGridDependencySynchronize) before it touches theta, v, the bf16
+ * copy, the batches or any other buffer of the call.  Contexts created with OMNI_NO_BULK_COPY
+ * launch only ordinary kernels and never signal early. */
 #define OMNI_BULK_COPY 8u
 #define OMNI_NO_BULK_COPY 16u
 
@@ -105,7 +115,7 @@ typedef struct omni_ctx omni_ctx;
 const char *omni_strerror(int status);
 
 /* Create a controller context with b_k = B / K (Algorithm 1, first line of Train).  Needs no GPU.
- * Errors: NULL, BAD_K, BAD_CONFIG, INFEASIBLE. */
+ * Errors: NULL, BAD_K, BAD_CONFIG, INFEASIBLE, NO_MEMORY. */
 int omni_create(const omni_config *cfg, omni_ctx **out);
 void omni_destroy(omni_ctx *ctx);
 
@@ -266,7 +276,9 @@ int omni_shard_range(uint64_t n, int32_t world, int32_t rank, uint64_t *begin, u
  * n elements each, owned by the caller; the call copies every host gradient into its staging
  * buffer on `stream`, runs the fused step, copies the squared gradient norm back, synchronises
  * the stream and stores it in *grad_sqnorm (host, may be NULL).
- * Errors: as omni_aggregate_bsp. */
+ * Errors: as omni_aggregate_bsp.  Unlike the other calls, a CUDA failure part-way (a copy or the
+ * launch refused by the runtime) can leave the staging buffers holding some of the new
+ * gradients; theta and v are only ever changed by the fused step itself. */
 int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                             const void *const *host_grads, const int32_t *b, float lr, float momentum,
                             float weight_decay, void *stream, double *grad_sqnorm);
@@ -279,7 +291,8 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
  * allocator lock, processes whose device memory has all been handed to a pool at start-up, and
  * latency-critical loops that ban calls which may synchronise the device, as cudaMalloc and
  * cudaFree may.  omni_aggregate_bsp allocates a small workspace on a context's first launch;
- * this function calls no cudaMalloc, cudaFree or any allocating routine, ever.  Its kernel's
+ * this function calls no cudaMalloc, cudaFree or other allocating routine (see "Warm-up" below
+ * for what the CUDA runtime does on its own the first time a kernel is used).  Its kernel's
  * scratch (per-CTA partial sums, the norm cell and a ticket counter, about 19 KB) is a fixed
  * array inside the library's device image: every GPU that loads the library holds it until the
  * process exits.
@@ -299,6 +312,15 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
  * First call: the first call on each device looks up the array's device address
  * (cudaGetSymbolAddress) with that device current; make that call before any stream capture.
  * It is not thread-safe against another first call on the same device.
+ * Warm-up: "never allocates" is what this function does itself.  The CUDA runtime loads a
+ * kernel's code, and whatever device memory that code needs, the first time the kernel is
+ * launched, and the first call for a combination of (device, gradient type, K, all buffers
+ * 32-byte aligned or not) also asks the runtime once for that kernel's occupancy.  A caller
+ * whose restriction covers the runtime's own lazy loading should therefore make one call per
+ * combination it will use (tiny buffers will do) before it enters the restricted region; every
+ * later call is one memset of 16 bytes, one kernel launch and, with grad_sqnorm_dev, one copy
+ * of 8 bytes, all asynchronous.
+ * flags: OMNI_UNSCALED_MEAN or 0; any other bit returns OMNI_ERR_BAD_CONFIG.
  * Errors: BAD_K, NULL, BAD_CONFIG, BAD_BATCH (some b_k < 1), ALIGN, TOO_LARGE, CUDA. */
 #define OMNI_NOALLOC_MAX_BUCKETS 8
 #define OMNI_NOALLOC_MAX_ELEMENTS (1ull << 31)

@@ -22,6 +22,7 @@ DEFAULT_FLAGS = 0  # OR-ed into every new context's flags (the tests use it to f
 OK = 0
 ERR_NULL, ERR_BAD_K, ERR_BAD_WORKER, ERR_BAD_BATCH, ERR_INFEASIBLE, ERR_BAD_MEASUREMENT = -1, -2, -3, -4, -5, -6
 ERR_ALIGN, ERR_BAD_TAU, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_CONFIG, ERR_TOO_LARGE = -7, -8, -9, -10, -11, -12
+ERR_NO_MEMORY = -13
 
 EXPORTS = (
     "omni_strerror", "omni_create", "omni_destroy", "omni_get_batches", "omni_set_batches",

@@ -11,7 +11,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libomni.so"
-SOURCES = [CSRC / "omni.cu", CSRC / "bulk_dispatch.cu", CSRC / "device_controller.cu", CSRC / "noalloc.cu",
+SOURCES = [CSRC / "omni.cu", CSRC / "register_dispatch.cu", CSRC / "bulk_dispatch.cu", CSRC / "device_controller.cu", CSRC / "noalloc.cu",
            CSRC / "controller.cpp", CSRC / "shard.cpp"]
 HEADERS = [CSRC / "kernels.cuh", CSRC / "tma_kernels.cuh", CSRC / "dispatch.h", CSRC / "controller.h",
            CSRC / "device_controller.h", PKG.parent / "include" / "omni.h"]

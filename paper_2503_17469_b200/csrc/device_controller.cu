@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(32) rebatch_kernel(DeviceCtl *c, const CtlCons
 template <typename G, int K> KernelInfo devlam_info()
 {
     constexpr TmaShape sh = tma_shape<G>(K);
-    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps, false, false, true>),
+    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps, false, true>),
             (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K), true};
 }
 
@@ -153,10 +153,7 @@ template <typename G> KernelInfo devlam_for(int K)
 {
     switch (K) {
 #define OMNI_CASE(k) case k: return devlam_info<G, k>();
-        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
-        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
-        OMNI_CASE(17) OMNI_CASE(18) OMNI_CASE(19) OMNI_CASE(20) OMNI_CASE(21) OMNI_CASE(22) OMNI_CASE(23) OMNI_CASE(24)
-        OMNI_CASE(25) OMNI_CASE(26) OMNI_CASE(27) OMNI_CASE(28) OMNI_CASE(29) OMNI_CASE(30) OMNI_CASE(31) OMNI_CASE(32)
+        OMNI_FOR_EACH_K(OMNI_CASE)
 #undef OMNI_CASE
     }
     return {};

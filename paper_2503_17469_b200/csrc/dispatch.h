@@ -1,5 +1,6 @@
 // Kernel selection shared by the translation units of the library (internal).
 #pragma once
+#include "../../include/omni.h"
 
 namespace omni {
 
@@ -15,6 +16,24 @@ struct KernelInfo {
     bool dependent_launch = false;  // the kernel waits for its predecessor itself (griddepcontrol.wait): launch it
                                     // with programmatic stream serialization so that its set-up overlaps that tail
 };
+
+// Kernels are templates on the worker count (the ordered FMA chain is unrolled at compile time), so
+// every selection by a run-time count is a switch over all of them.  The case lists live here,
+// once: X(k) for every worker count / every length of a queue of asynchronous arrivals.
+#define OMNI_FOR_EACH_K(X)                                                                                  \
+    X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16)                  \
+    X(17) X(18) X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32)
+#define OMNI_FOR_EACH_QUEUE(X) \
+    X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16)
+static_assert(OMNI_MAX_K == 32 && OMNI_MAX_ASP_BATCH == 16, "the case lists above cover 1..32 and 1..16");
+
+// Register-staged kernels (register_dispatch.cu): the synchronous step for K workers, the
+// asynchronous apply of one arrival and of M queued arrivals, the push with overwrite.
+// wide = every buffer is 32-byte aligned (256-bit loads and stores), else 128-bit.
+KernelInfo bsp_kernel(int dtype, int K, bool wide);
+KernelInfo seq_kernel(int dtype, int M, bool wide);
+KernelInfo asp_kernel(int dtype, bool wide, bool momentum);
+KernelInfo overwrite_kernel(int dtype, bool wide);
 
 // Bulk-copy ring kernels (bulk_dispatch.cu): the synchronous step for K workers, and the
 // asynchronous apply of M queued arrivals (M = 1: a single arrival; M <= OMNI_MAX_ASP_BATCH).

@@ -22,6 +22,7 @@
 #include <cmath>
 #include <cstring>
 
+#include "dispatch.h"
 #include "kernels.cuh"
 
 namespace omni {
@@ -34,6 +35,7 @@ static __device__ __align__(256) unsigned long long noalloc_scratch[(sizeof(Work
 constexpr int kMaxDevices = 64;
 Workspace *g_scratch_addr[kMaxDevices] = {};  // device address of noalloc_scratch, per device
 int g_sm_count[kMaxDevices] = {};
+int g_grid[kMaxDevices][2][2][OMNI_MAX_K + 1] = {};  // [device][dtype][256-bit][K]: persistent grid, 0 = not asked yet
 
 // Once per device, with that device current: resolve the device address of the scratch array.
 cudaError_t scratch_for_current_device(Workspace **out, int *sms)
@@ -57,36 +59,6 @@ cudaError_t scratch_for_current_device(Workspace **out, int *sms)
     return cudaSuccess;
 }
 
-struct Pick {
-    const void *fn = nullptr;
-    int threads = 0, ctas_per_sm = 0;
-    unsigned long long tile = 0;
-};
-
-template <typename G, int K, bool WIDE> Pick pick_one()
-{
-    constexpr Shape sh = bsp_shape<G>(K);
-    return {reinterpret_cast<const void *>(&bsp_fused_kernel<G, K, sh.threads, sh.chunks, WIDE>), sh.threads,
-            sh.ctas_per_sm, (unsigned long long)sh.threads * Geo<G, WIDE>::E * sh.chunks};
-}
-template <typename G, bool WIDE> Pick pick_k(int K)
-{
-    switch (K) {
-#define OMNI_CASE(k) case k: return pick_one<G, k, WIDE>();
-        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
-        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
-        OMNI_CASE(17) OMNI_CASE(18) OMNI_CASE(19) OMNI_CASE(20) OMNI_CASE(21) OMNI_CASE(22) OMNI_CASE(23) OMNI_CASE(24)
-        OMNI_CASE(25) OMNI_CASE(26) OMNI_CASE(27) OMNI_CASE(28) OMNI_CASE(29) OMNI_CASE(30) OMNI_CASE(31) OMNI_CASE(32)
-#undef OMNI_CASE
-    }
-    return {};
-}
-Pick pick(int dtype, int K, bool wide)
-{
-    if (dtype == OMNI_BF16) return wide ? pick_k<__nv_bfloat16, true>(K) : pick_k<__nv_bfloat16, false>(K);
-    return wide ? pick_k<float, true>(K) : pick_k<float, false>(K);
-}
-
 bool is_aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 }  // namespace
@@ -102,6 +74,7 @@ extern "C" int omni_aggregate_bsp_noalloc(int32_t K, const omni_bucket *buckets,
     if (!b || (n_buckets > 0 && !buckets)) return OMNI_ERR_NULL;
     if (n_buckets < 0 || (grad_dtype != OMNI_F32 && grad_dtype != OMNI_BF16) || !std::isfinite(momentum))
         return OMNI_ERR_BAD_CONFIG;
+    if (flags & ~uint32_t(OMNI_UNSCALED_MEAN)) return OMNI_ERR_BAD_CONFIG;   // no other flag means anything here
     int64_t total_b = 0;
     for (int k = 0; k < K; ++k) {
         if (b[k] < 1) return OMNI_ERR_BAD_BATCH;
@@ -133,13 +106,19 @@ extern "C" int omni_aggregate_bsp_noalloc(int32_t K, const omni_bucket *buckets,
     if (scratch_for_current_device(&ws, &sms) != cudaSuccess) return OMNI_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    const Pick pk = pick(grad_dtype, K, wide);
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pk.fn, pk.threads, 0) != cudaSuccess) return OMNI_ERR_CUDA;
-    if (per_sm < 1) per_sm = 1;
-    if (per_sm > pk.ctas_per_sm) per_sm = pk.ctas_per_sm;
-    int grid = sms * per_sm;
-    if (grid > kMaxGrid) grid = kMaxGrid;
+    const KernelInfo pk = bsp_kernel(grad_dtype, K, wide);   // the register-staged synchronous kernel
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return OMNI_ERR_CUDA;
+    // persistent grid of this kernel on this device, asked of the runtime once and kept
+    int &cached = g_grid[dev][grad_dtype][wide ? 1 : 0][K];
+    if (cached == 0) {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pk.fn, pk.threads, 0) != cudaSuccess) return OMNI_ERR_CUDA;
+        if (per_sm < 1) per_sm = 1;
+        if (pk.ctas_per_sm > 0 && per_sm > pk.ctas_per_sm) per_sm = pk.ctas_per_sm;
+        cached = sms * per_sm > kMaxGrid ? kMaxGrid : sms * per_sm;
+    }
+    int grid = cached;
 
     BspParams p;
     std::memset(&p, 0, sizeof p);

@@ -51,77 +51,6 @@ namespace {
         }                                            \
     } while (0)
 
-template <typename G, int K, bool WIDE> KernelInfo bsp_info()
-{
-    constexpr Shape sh = bsp_shape<G>(K);
-    return {reinterpret_cast<KernelFn>(&bsp_fused_kernel<G, K, sh.threads, sh.chunks, WIDE>), sh.threads,
-            sh.ctas_per_sm, (unsigned long long)sh.threads * Geo<G, WIDE>::E * sh.chunks};
-}
-
-template <typename G, bool WIDE> KernelInfo bsp_kernel_for(int K)
-{
-    switch (K) {
-#define OMNI_CASE(k) case k: return bsp_info<G, k, WIDE>();
-        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
-        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
-        OMNI_CASE(17) OMNI_CASE(18) OMNI_CASE(19) OMNI_CASE(20) OMNI_CASE(21) OMNI_CASE(22) OMNI_CASE(23) OMNI_CASE(24)
-        OMNI_CASE(25) OMNI_CASE(26) OMNI_CASE(27) OMNI_CASE(28) OMNI_CASE(29) OMNI_CASE(30) OMNI_CASE(31) OMNI_CASE(32)
-#undef OMNI_CASE
-    }
-    return {};
-}
-
-KernelInfo bsp_kernel(int dtype, int K, bool wide)
-{
-    if (dtype == OMNI_BF16) return wide ? bsp_kernel_for<__nv_bfloat16, true>(K) : bsp_kernel_for<__nv_bfloat16, false>(K);
-    return wide ? bsp_kernel_for<float, true>(K) : bsp_kernel_for<float, false>(K);
-}
-
-// Batched asynchronous apply, M = arrivals in the batch; launch shape as the synchronous kernel with K = M.
-template <typename G, int M, bool WIDE> KernelInfo seq_info()
-{
-    constexpr Shape sh = bsp_shape<G>(M);
-    return {reinterpret_cast<KernelFn>(&asp_batch_kernel<G, M, sh.threads, sh.chunks, WIDE>), sh.threads,
-            sh.ctas_per_sm, (unsigned long long)sh.threads * Geo<G, WIDE>::E * sh.chunks};
-}
-template <typename G, bool WIDE> KernelInfo seq_kernel_for(int M)
-{
-    switch (M) {
-#define OMNI_CASE(k) case k: return seq_info<G, k, WIDE>();
-        OMNI_CASE(1) OMNI_CASE(2) OMNI_CASE(3) OMNI_CASE(4) OMNI_CASE(5) OMNI_CASE(6) OMNI_CASE(7) OMNI_CASE(8)
-        OMNI_CASE(9) OMNI_CASE(10) OMNI_CASE(11) OMNI_CASE(12) OMNI_CASE(13) OMNI_CASE(14) OMNI_CASE(15) OMNI_CASE(16)
-#undef OMNI_CASE
-    }
-    return {};
-}
-KernelInfo seq_kernel(int dtype, int M, bool wide)
-{
-    if (dtype == OMNI_BF16) return wide ? seq_kernel_for<__nv_bfloat16, true>(M) : seq_kernel_for<__nv_bfloat16, false>(M);
-    return wide ? seq_kernel_for<float, true>(M) : seq_kernel_for<float, false>(M);
-}
-
-template <typename G, bool WIDE> KernelInfo overwrite_info()
-{
-    return {reinterpret_cast<KernelFn>(&asp_overwrite_kernel<G, kAspThreads, kAspChunks, WIDE>), kAspThreads,
-            asp_ctas_per_sm(false), (unsigned long long)kAspThreads * Geo<G, WIDE>::E * kAspChunks};
-}
-KernelInfo overwrite_kernel(int dtype, bool wide)
-{
-    if (dtype == OMNI_BF16) return wide ? overwrite_info<__nv_bfloat16, true>() : overwrite_info<__nv_bfloat16, false>();
-    return wide ? overwrite_info<float, true>() : overwrite_info<float, false>();
-}
-
-template <typename G, bool WIDE> KernelInfo asp_info(bool momentum)
-{
-    return {reinterpret_cast<KernelFn>(&asp_apply_kernel<G, kAspThreads, kAspChunks, WIDE>), kAspThreads,
-            asp_ctas_per_sm(momentum), (unsigned long long)kAspThreads * Geo<G, WIDE>::E * kAspChunks};
-}
-KernelInfo asp_kernel(int dtype, bool wide, bool momentum)
-{
-    if (dtype == OMNI_BF16) return wide ? asp_info<__nv_bfloat16, true>(momentum) : asp_info<__nv_bfloat16, false>(momentum);
-    return wide ? asp_info<float, true>(momentum) : asp_info<float, false>(momentum);
-}
-
 // First kernel-launching call of a context: bind to the current device, allocate the workspace.
 int ensure_device(omni_ctx *ctx)
 {
@@ -333,6 +262,7 @@ const char *omni_strerror(int s)
         case OMNI_ERR_TIMEOUT: return "device-side wait ran out";
         case OMNI_ERR_BAD_CONFIG: return "invalid configuration or argument";
         case OMNI_ERR_TOO_LARGE: return "size beyond the stated maximum";
+        case OMNI_ERR_NO_MEMORY: return "host memory allocation failed";
     }
     return "unknown status";
 }
@@ -343,7 +273,7 @@ int omni_create(const omni_config *cfg, omni_ctx **out)
     const int rc = BatchController::validate(*cfg);
     if (rc != OMNI_OK) return rc;
     omni_ctx *ctx = new (std::nothrow) omni_ctx(*cfg);
-    if (!ctx) return OMNI_ERR_CUDA;
+    if (!ctx) return OMNI_ERR_NO_MEMORY;
     ctx->tally.tau_max = 0;
     *out = ctx;
     return OMNI_OK;

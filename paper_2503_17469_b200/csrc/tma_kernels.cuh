@@ -136,15 +136,14 @@ template <typename G> __host__ __device__ constexpr unsigned tma_smem_bytes(int 
     return tma_ring_bytes(tma_shape<G>(K), K, int(sizeof(G)));
 }
 
-template <typename G, int K, int TILE, int STAGES, int NCW, bool WIDE, bool SEQ = false, bool DEVLAM = false, bool OVW = false>
+template <typename G, int K, int TILE, int STAGES, int NCW, bool SEQ = false, bool DEVLAM = false, bool OVW = false>
 __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_constant__ BspParams p)
 {
     constexpr int THREADS = (NCW + 1) * 32;
     constexpr int NCT = NCW * 32;                       // consumer threads
     constexpr int V = 16 / int(sizeof(G));              // elements per 16-byte gradient vector
-    constexpr int NV = WIDE ? 2 : 1;                    // vectors per work item (WIDE: 32-byte global stores)
+    constexpr int NV = 1;                               // gradient vectors per work item
     constexpr int E = V * NV;                           // elements per work item
-    constexpr int SW = WIDE ? 8 : 4;                    // words per theta/v store
     constexpr unsigned GB = TILE * sizeof(G);           // bytes of one gradient tile
     constexpr unsigned FB = TILE * 4;                   // bytes of a theta or v tile
     constexpr unsigned SB = K * GB + 2 * FB;            // bytes of one stage
@@ -297,13 +296,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32) bsp_tma_kernel(const __grid_co
                         }
                     }
                     const unsigned long long off = base + (unsigned long long)j * E;
-                    if constexpr (WIDE) {
-                        store_floats<SW, E / SW>(bd.theta + off, th);
-                        if (has_v) store_floats<SW, E / SW>(bd.v + off, vv);
-                    } else {
-                        store_floats_policy<E>(bd.theta + off, th, pol_keep);
-                        if (has_v) store_floats_policy<E>(bd.v + off, vv, pol_keep);
-                    }
+                    store_floats_policy<E>(bd.theta + off, th, pol_keep);
+                    if (has_v) store_floats_policy<E>(bd.v + off, vv, pol_keep);
                     if (has_lp) store_lp<E / 2>(bd.lp + off, th);
                     if constexpr (OVW) { if (cpy) store_floats<4, E / 4>(cpy + off, th); }
                 }

@@ -546,60 +546,102 @@ def test_vgg16_config_shrunk_with_interference_phase():
     _bsp_config_run("vgg16", 50, numel_cap=5000)
 
 
-def _sample_blocks(total, rng, n_blocks=48, width=4096):
-    starts = sorted(int(s) for s in rng.integers(0, max(total - width, 1), n_blocks))
-    return [(s, min(s + width, total)) for s in starts]
+def _chunks(lay, width=1 << 22):
+    """Element ranges that tile every bucket of the layout, at most ``width`` elements each."""
+    for bk in lay.buckets:
+        for s in range(bk.start, bk.start + bk.n, width):
+            yield s, min(s + width, bk.start + bk.n)
 
 
-def test_vgg16_config_full_size_sampled():
-    """K=32, 138M parameters, 7 buckets: two steps at full size; the oracle recomputes sampled
-    blocks (the rules are element-wise, so a block needs only its own inputs) including every
-    bucket's first and last elements; the squared norm is checked against its expectation for
-    i.i.d. gradients, sigma^2 * sum(lambda^2) * P."""
+def _oracle_threads():
+    import os
+
+    return max(1, min(16, len(os.sched_getaffinity(0))))
+
+
+def test_vgg16_config_full_size_every_element():
+    """K=32, 138M parameters, 7 buckets: two steps at full size with a re-batch before each (the
+    configuration re-batches every step), every element of theta and v against the oracle and the
+    squared norm of both steps against the oracle's sums.  The rules are element-wise, so the
+    oracle walks the buckets in ranges of 4M elements (bounded host memory), several ranges at a
+    time on the host cores."""
+    from concurrent.futures import ThreadPoolExecutor
+
     cfg = W.config("vgg16")
     buf = W.make_buffers(cfg, DEV)
     lay = buf.layout
     o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
+    ora = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband)
     gen = torch.Generator().manual_seed(cfg.seed)
-    T = W.draw_throughputs(cfg.K, gen, cfg.ratio)
-    b, _ = o.rebatch(T)
+    base = W.draw_throughputs(cfg.K, gen, cfg.ratio)
     bs = B.BucketSet.from_flat(lay, buf.theta, buf.grads, buf.v)
-    rng = np.random.default_rng(cfg.seed)
-    blocks = _sample_blocks(lay.total, rng)
-    for bk in lay.buckets:
-        blocks += [(bk.start, min(bk.start + 300, bk.start + bk.n)), (max(bk.start, bk.start + bk.n - 300), bk.start + bk.n)]
-    snap = [(to_np(buf.theta[s:e]), to_np(buf.v[s:e]), [to_np(g[s:e]) for g in buf.grads]) for s, e in blocks]
-    for _ in range(2):
+    th0, v0 = buf.theta.cpu(), buf.v.cpu()          # the state before the first step
+    steps, batches, sq_gpu = 2, [], []
+    for step in range(steps):
+        T = W.jitter_throughputs(W.interference(base, step), gen)
+        b, _ = o.rebatch(T)
+        assert b == ora.rebatch(T)[0].tolist() and sum(b) == cfg.global_batch
+        batches.append(b)
         o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum)
-    for (s, e), (th_o, v_o, g_np) in zip(blocks, snap):
-        for _ in range(2):
-            O.bsp_step_f32(g_np, b, th_o, v_o, cfg.lr, cfg.momentum, 0.0)
-        assert np.array_equal(to_np(buf.theta[s:e]), th_o), (s, e)
-        assert np.array_equal(to_np(buf.v[s:e]), v_o), (s, e)
-    lam = O.bsp_weights(b)[0]
-    expect = cfg.grad_std ** 2 * float((lam ** 2).sum()) * cfg.P
-    assert abs(o.stats().grad_sqnorm - expect) <= 0.01 * expect
+        sq_gpu.append(o.stats().grad_sqnorm)
+    assert batches[0] != batches[1]
+    th1, v1 = buf.theta.cpu(), buf.v.cpu()
+
+    def one(rng):
+        s, e = rng
+        g_np = [to_np(g[s:e]) for g in buf.grads]
+        th_o, v_o = th0[s:e].numpy().copy(), v0[s:e].numpy().copy()
+        sq = [O.bsp_step_f32(g_np, b, th_o, v_o, cfg.lr, cfg.momentum, 0.0) for b in batches]
+        ok = np.array_equal(th1[s:e].numpy(), th_o) and np.array_equal(v1[s:e].numpy(), v_o)
+        return ok, sq
+
+    covered = 0
+    sq_o = [0.0] * steps
+    with ThreadPoolExecutor(max_workers=_oracle_threads()) as ex:
+        for (s, e), (ok, sq) in zip(_chunks(lay), ex.map(one, _chunks(lay))):
+            assert ok, (s, e)
+            covered += e - s
+            for i in range(steps):
+                sq_o[i] += sq[i]
+    assert covered == sum(bk.n for bk in lay.buckets) >= cfg.P
+    for got, want in zip(sq_gpu, sq_o):
+        assert abs(got - want) <= SQNORM_RTOL * want
 
 
-def test_resnet50_asp_full_size_sampled():
-    """25.6M parameters, 20 arrivals at full size against the oracle on sampled blocks."""
+def test_resnet50_asp_full_size_every_element():
+    """25.6M parameters, 20 arrivals with controller feedback at full size: every element of the
+    server parameters against the oracle."""
+    from concurrent.futures import ThreadPoolExecutor
+
     cfg = W.config("resnet50_asp")
     buf = W.make_buffers(cfg, DEV)
     lay = buf.layout
     o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, 1.0, B.ASP)
+    ora = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, 1.0, O.MODE_ASP)
     bs = B.BucketSet.from_flat(lay, buf.theta, buf.grads)
-    rng = np.random.default_rng(cfg.seed)
-    blocks = _sample_blocks(lay.total, rng)
-    for bk in lay.buckets:
-        blocks += [(bk.start, bk.start + 300), (bk.start + bk.n - 300, bk.start + bk.n)]
-    snap = [(to_np(buf.theta[s:e]), [to_np(g[s:e]) for g in buf.grads]) for s, e in blocks]
+    th0 = buf.theta.cpu()
     events = []
-    _asp_stream(cfg, 20, lambda k, bu, tau: (events.append((k, bu, tau)), o.apply_asp(bs, k, bu, tau, cfg.lr)),
-                o.asp_report, cfg.seed)
-    for (s, e), (th_o, g_np) in zip(blocks, snap):
+    t_lib = _asp_stream(cfg, 20, lambda k, bu, tau: (events.append((k, bu, tau)), o.apply_asp(bs, k, bu, tau, cfg.lr)),
+                        o.asp_report, cfg.seed)
+    t_ora = _asp_stream(cfg, 20, lambda k, bu, tau: None, ora.asp_report, cfg.seed)
+    assert t_lib == t_ora
+    th1 = buf.theta.cpu()
+    g_host = [g.cpu() for g in buf.grads]
+
+    def one(rng):
+        s, e = rng
+        th_o = th0[s:e].numpy().copy()
         for k, bu, tau in events:
-            O.asp_apply_f32(g_np[k], bu, cfg.global_batch, th_o, None, cfg.lr, 0.0, 0.0)
-        assert np.array_equal(to_np(buf.theta[s:e]), th_o), (s, e)
+            O.asp_apply_f32(g_host[k][s:e].numpy(), bu, cfg.global_batch, th_o, None, cfg.lr, 0.0, 0.0)
+        return np.array_equal(th1[s:e].numpy(), th_o)
+
+    covered = 0
+    with ThreadPoolExecutor(max_workers=_oracle_threads()) as ex:
+        for (s, e), ok in zip(_chunks(lay), ex.map(one, _chunks(lay))):
+            assert ok, (s, e)
+            covered += e - s
+    assert covered == sum(bk.n for bk in lay.buckets) >= cfg.P
+    assert o.stats().arrivals == 20
 
 
 def test_bucket_longer_than_32_bit_indices():

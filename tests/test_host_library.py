@@ -25,7 +25,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_strerror_covers_all_codes():
     L = B.lib()
-    for code in range(0, -13, -1):
+    for code in range(0, -14, -1):
         assert L.omni_strerror(code) and L.omni_strerror(code) != b"unknown status"
     assert L.omni_strerror(-99) == b"unknown status"
 
