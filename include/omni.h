@@ -21,7 +21,10 @@
  *   - A context is not thread-safe.  It owns a small device workspace (per-block partial sums
  *     and the gradient-norm cell, a few tens of KB) that is allocated by the first call that
  *     launches a kernel and freed by omni_destroy; calls on different streams that share a
- *     context and overlap on the GPU race on it.
+ *     context and overlap on the GPU race on it.  The synchronous step leaves one partial sum of
+ *     the squared gradient norm per thread block there; they are added up, in a fixed order, by
+ *     a one-warp kernel that omni_get_stats and omni_aggregate_bsp_host enqueue, so a step that
+ *     nobody asks the norm of pays nothing for it.
  *   - OMNI_MAX_K = 32 workers.
  */
 #ifndef OMNI_H_
@@ -60,6 +63,14 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
 #define OMNI_UNSCALED_MEAN 1u   /* lambda_k = 1/K: the unweighted arm of the paper's "weighted aggregation" table */
 #define OMNI_ASP_NO_LR_SCALE 2u /* eta_k = eta: the "w/o LR scaling" arm of the paper's ASP table */
 #define OMNI_INPUT_IS_TIME 4u   /* measurements are compute times t_k instead of throughputs T_k */
+/* Global-batch rule, second reading.  Eq. 8 subtracts the same Delta B / K from every worker
+ * (the default); the sentence after it (Sec. III-B, "Control Stability") speaks of reducing the
+ * adjusted batches "proportionately".  With this flag the synchronous re-batch renormalises the
+ * real-valued getBsz results c_k of all workers, c_k <- c_k * B / sum_i c_i, before the rounding
+ * step, and the unit steps of the default rule only close what rounding and the bounds leave.
+ * From equal batches without dead-band and bounds this gives B * T_k / sum(T) in one step
+ * (Eq. 4a with the throughputs as capacities).  Ignored in asynchronous mode. */
+#define OMNI_CONSERVE_MULTIPLICATIVE 32u
 /* Kernel family.  By default the device calls stage their inputs through shared memory with
  * bulk (TMA) copies and an mbarrier ring; register-staged 128/256-bit-load kernels exist for
  * every call as well (and serve omni_aggregate_bsp_noalloc).  The ring
@@ -293,20 +304,21 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
  * cudaFree may.  omni_aggregate_bsp allocates a small workspace on a context's first launch;
  * this function calls no cudaMalloc, cudaFree or other allocating routine (see "Warm-up" below
  * for what the CUDA runtime does on its own the first time a kernel is used).  Its kernel's
- * scratch (per-CTA partial sums, the norm cell and a ticket counter, about 19 KB) is a fixed
+ * scratch (one partial sum of the squared norm per CTA, about 19 KB) is a fixed
  * array inside the library's device image: every GPU that loads the library holds it until the
  * process exits.
  *
  * It takes no context: K, the batches and the flags (OMNI_UNSCALED_MEAN) come as arguments and
  * lambda_k = b_k / sum b.  Arithmetic, layouts and alignment rules are those of
  * omni_aggregate_bsp.  grad_sqnorm_dev (DEVICE pointer, 8-byte aligned, may be NULL) receives
- * the squared norm of the aggregate by a copy enqueued after the kernel.  Enqueues on `stream`,
- * does not synchronise.
+ * the squared norm of the aggregate from a one-warp kernel enqueued after the step (it adds the
+ * partial sums in a fixed order; with NULL it is not launched).  Enqueues on `stream`, does not
+ * synchronise.
  *
  * Limits: at most OMNI_NOALLOC_MAX_BUCKETS non-empty buckets and OMNI_NOALLOC_MAX_ELEMENTS
  * elements in total; more returns OMNI_ERR_TOO_LARGE and does nothing.
  * Sharing: all calls on one device use the same array, which keeps the previous call's
- * contents; the function zeroes the cells that must start at zero before each launch.  Calls
+ * contents; no cell has to start at zero (each launch overwrites every cell it later reads).  Calls
  * whose kernels overlap on the GPU (issued on different streams without ordering) race on it
  * and give wrong norms: keep them on one stream or order them with events.
  * First call: the first call on each device looks up the array's device address
@@ -318,8 +330,8 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
  * 32-byte aligned or not) also asks the runtime once for that kernel's occupancy.  A caller
  * whose restriction covers the runtime's own lazy loading should therefore make one call per
  * combination it will use (tiny buffers will do) before it enters the restricted region; every
- * later call is one memset of 16 bytes, one kernel launch and, with grad_sqnorm_dev, one copy
- * of 8 bytes, all asynchronous.
+ * later call is one kernel launch and, with grad_sqnorm_dev, a second one-warp launch, both
+ * asynchronous.
  * flags: OMNI_UNSCALED_MEAN or 0; any other bit returns OMNI_ERR_BAD_CONFIG.
  * Errors: BAD_K, NULL, BAD_CONFIG, BAD_BATCH (some b_k < 1), ALIGN, TOO_LARGE, CUDA. */
 #define OMNI_NOALLOC_MAX_BUCKETS 8

@@ -17,6 +17,7 @@ TAU_BINS = 33
 BSP, ASP = 0, 1
 F32, BF16 = 0, 1
 UNSCALED_MEAN, ASP_NO_LR_SCALE, INPUT_IS_TIME, BULK_COPY, NO_BULK_COPY = 1, 2, 4, 8, 16
+CONSERVE_MULTIPLICATIVE = 32
 DEFAULT_FLAGS = 0  # OR-ed into every new context's flags (the tests use it to force a kernel family)
 
 OK = 0

@@ -21,6 +21,12 @@ __global__ void expire_wait_kernel(Workspace *ws, unsigned attempts)
 }
 
 
+__global__ void __launch_bounds__(32) sqnorm_finalize_kernel(const Workspace *ws, int slots, double *out)
+{
+    const double s = ordered_partial_sum(ws->partials, slots);
+    if (threadIdx.x == 0) *out = s;
+}
+
 template <typename G, int K> KernelInfo bulk_info()
 {
     constexpr TmaShape sh = tma_shape<G>(K);
@@ -71,6 +77,12 @@ KernelInfo bulk_overwrite_kernel(int dtype)
 
 KernelInfo bulk_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bulk_for<__nv_bfloat16>(K) : bulk_for<float>(K); }
 KernelInfo bulk_seq_kernel(int dtype, int M) { return dtype == OMNI_BF16 ? bulk_seq_for<__nv_bfloat16>(M) : bulk_seq_for<float>(M); }
+
+int launch_sqnorm_finalize(void *workspace, int slots, double *out, void *stream)
+{
+    sqnorm_finalize_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const Workspace *>(workspace), slots, out);
+    return int(cudaGetLastError());
+}
 
 int launch_expire_wait(void *workspace, unsigned attempts, void *stream)
 {

@@ -85,7 +85,7 @@ BatchController::Proposal BatchController::propose(int32_t b, double t, double t
     if (rel >= cfg_.deadband)
         chosen = target < double(cfg_.b_min) ? double(cfg_.b_min)
                : target > double(cfg_.b_max) ? double(cfg_.b_max) : target;
-    return {target, to_integer(chosen)};
+    return {target, chosen, to_integer(chosen)};
 }
 
 // Eq. 8 on integers with bounds.  The uniform shift Delta B / K is applied in blocks of whole
@@ -134,7 +134,20 @@ int BatchController::rebatch(const double *measured, int32_t *new_b, int32_t *ch
     const double tbar = total / double(K);
 
     std::array<int32_t, OMNI_MAX_K> n{};
-    for (int k = 0; k < K; ++k) n[k] = propose(batch_[k], t[k], tbar).rounded;
+    if (cfg_.mode == OMNI_BSP && (cfg_.flags & OMNI_CONSERVE_MULTIPLICATIVE)) {
+        // the other reading of the sentence after Eq. 8: renormalise the real-valued getBsz
+        // results to the global batch before the rounding step
+        std::array<double, OMNI_MAX_K> c{};
+        double csum = 0.0;
+        for (int k = 0; k < K; ++k) c[k] = propose(batch_[k], t[k], tbar).chosen;
+        for (int k = 0; k < K; ++k) csum += c[k];
+        for (int k = 0; k < K; ++k) {
+            const double scaled_up = c[k] * double(cfg_.global_batch);
+            n[k] = to_integer(scaled_up / csum);
+        }
+    } else {
+        for (int k = 0; k < K; ++k) n[k] = propose(batch_[k], t[k], tbar).rounded;
+    }
     if (cfg_.mode == OMNI_BSP) {
         const int rc = close_gap(n);
         if (rc != OMNI_OK) return rc;

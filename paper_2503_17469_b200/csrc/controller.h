@@ -32,7 +32,7 @@ public:
     void import_state(const int32_t *b, const double *time, const int32_t *seen);
 
 private:
-    struct Proposal { double real; int32_t rounded; };
+    struct Proposal { double real; double chosen; int32_t rounded; };   // b* of Eq. 6b; after dead-band and bounds; as an integer
     double to_time(int32_t b, double measured) const;
     double smoothed(int k, double t, const std::array<double, OMNI_MAX_K> &cur,
                     const std::array<bool, OMNI_MAX_K> &seen) const;

@@ -81,13 +81,27 @@ __global__ void __launch_bounds__(32) rebatch_kernel(DeviceCtl *c, const CtlCons
 
     // getBsz: Eq. 6b, dead-band (Eq. 7), bounds, one rounding to an integer (half up)
     int32_t n = 0;
+    double chosen = 0.0;
     if (on) {
         const double throughput = __ddiv_rn(bd, s);
         const double error = __dsub_rn(s, tbar);
         const double target = __dsub_rn(bd, __dmul_rn(throughput, error));
         const double rel = fabs(__ddiv_rn(__dsub_rn(target, bd), target));
-        double chosen = bd;
+        chosen = bd;
         if (rel >= cc.deadband) chosen = target < lo ? lo : target > hi ? hi : target;
+    }
+    if (cc.mode == OMNI_BSP && (cc.flags & OMNI_CONSERVE_MULTIPLICATIVE)) {
+        // the other reading of the sentence after Eq. 8: renormalise the real-valued results to the
+        // global batch before rounding (their sum in ascending k by every lane, as on the host)
+        double csum = 0.0;
+#pragma unroll
+        for (int j = 0; j < OMNI_MAX_K; ++j) {
+            const double cj = __shfl_sync(kFull, chosen, j);
+            if (j < cc.K) csum = __dadd_rn(csum, cj);
+        }
+        if (on) chosen = __ddiv_rn(__dmul_rn(chosen, double(cc.B)), csum);
+    }
+    if (on) {
         double r = floor(__dadd_rn(chosen, 0.5));
         r = r < lo ? lo : r;
         r = hi < r ? hi : r;

@@ -50,6 +50,11 @@ KernelInfo bulk_overwrite_kernel(int dtype);
 // the bandwidth).
 bool bulk_preferred(int dtype, int streams);
 
+// Enqueues the one-warp kernel that adds the first `slots` per-CTA partials of the workspace in
+// index order and stores the sum in *out (a device address: the workspace's own cell, or the
+// caller's); returns the cudaError_t as int.
+int launch_sqnorm_finalize(void *workspace, int slots, double *out, void *stream);
+
 // Launches the bounded-wait diagnostic kernel (bulk_dispatch.cu); returns the cudaError_t as int.
 int launch_expire_wait(void *workspace, unsigned attempts, void *stream);
 

@@ -6,14 +6,13 @@
 // pool, and real-time loops that forbid anything that may synchronise the device (cudaMalloc
 // and cudaFree may).  The regular entry point allocates a small workspace the first time a
 // context launches a kernel; this one never allocates.  The kernel's scratch -- one squared-norm
-// partial per CTA, the result cell and the ticket counter -- lives in a fixed array in device
-// memory that is part of the library image, so every GPU that loads the library carries these
-// ~19 KB until the process exits.
+// partial per CTA -- lives in a fixed array in device memory that is part of the library image,
+// so every GPU that loads the library carries these ~19 KB until the process exits.
 //
 // Consequences the caller has to know (also stated in omni.h):
-//   - the array is shared by every call on that device and keeps the last call's contents; the
-//     entry point clears the cells that must start at zero before each launch, but two calls
-//     whose kernels overlap on the GPU (different streams) race on it;
+//   - the array is shared by every call on that device and keeps the last call's contents;
+//     nothing in it has to start at zero (a launch overwrites every cell that is read after
+//     it), but two calls whose kernels overlap on the GPU (different streams) race on it;
 //   - the first call on each device looks up the array's device address; make that first call
 //     outside any stream capture;
 //   - sizes are bounded (OMNI_NOALLOC_MAX_BUCKETS, OMNI_NOALLOC_MAX_ELEMENTS).
@@ -142,12 +141,11 @@ extern "C" int omni_aggregate_bsp_noalloc(int32_t K, const omni_bucket *buckets,
     p.ws = ws;
     if (tiles < (unsigned long long)grid) grid = tiles < 1 ? 1 : int(tiles);
 
-    // the array keeps whatever the previous call left: the ticket and the result cell start at zero
-    if (cudaMemsetAsync(&ws->sqnorm, 0, sizeof(double) + 2 * sizeof(unsigned int), s) != cudaSuccess) return OMNI_ERR_CUDA;
+    // The array keeps whatever the previous call left.  Nothing in it has to start at zero: every
+    // CTA of this launch overwrites its own partial-sum slot (p.accumulate == 0), and the sum
+    // below reads exactly the slots this launch wrote.
     void *args[] = {&p};
     if (cudaLaunchKernel(pk.fn, dim3(grid), dim3(pk.threads), args, 0, s) != cudaSuccess) return OMNI_ERR_CUDA;
-    if (grad_sqnorm_dev &&
-        cudaMemcpyAsync(grad_sqnorm_dev, &ws->sqnorm, sizeof(double), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
-        return OMNI_ERR_CUDA;
+    if (grad_sqnorm_dev && launch_sqnorm_finalize(ws, grid, grad_sqnorm_dev, stream) != 0) return OMNI_ERR_CUDA;
     return OMNI_OK;
 }

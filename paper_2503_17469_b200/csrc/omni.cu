@@ -27,6 +27,7 @@ struct omni_ctx {
     int last_cuda = 0;
     uint64_t launches = 0;
     unsigned sweep = 0;              // calls that walked the parameters so far (parity = sweep direction)
+    int sq_slots = 0;                // per-CTA norm partials the last synchronous step left in the workspace
     omni::DeviceCtl *dctl = nullptr; // device copy of the controller (omni_ctl_to_device), or null
     omni::DeviceCtl dctl_stage{};    // host staging for its uploads and downloads
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
@@ -171,6 +172,19 @@ int launch(omni_ctx *ctx, const KernelInfo &ki, int grid, void *params, cudaStre
     return OMNI_OK;
 }
 
+// The squared norm of the last synchronous step: add its per-CTA partials up on the device.
+int finalize_sqnorm(omni_ctx *ctx, cudaStream_t stream)
+{
+    if (ctx->sq_slots == 0) return OMNI_OK;
+    const int e = launch_sqnorm_finalize(ctx->ws, ctx->sq_slots, &ctx->ws->sqnorm, stream);
+    if (e != 0) {
+        ctx->last_cuda = e;
+        return OMNI_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return OMNI_OK;
+}
+
 // Eq. 4b: lambda_k = b_k / sum b, evaluated in double and rounded once to float.
 double fill_weights(const omni_ctx *ctx, const int32_t *b, float *lam)
 {
@@ -203,7 +217,7 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
     const unsigned long long tile = ki.tile;
 
     BspParams p;
-    int launched = 0, i = 0;
+    int launched = 0, i = 0, slots = 0;
     while (i < n_buckets || launched == 0) {
         std::memset(&p, 0, sizeof p);
         unsigned long long tiles = 0;
@@ -222,7 +236,7 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
         p.lam_dev = lam_dev;
         p.lr = lr; p.mu = mu; p.wd = wd;
         p.nb = nb;
-        p.accumulate = launched > 0;
+        p.accumulate = slots;
         p.reverse = int(ctx->sweep & 1u);
         p.tiles = tiles;
         p.ws = ctx->ws;
@@ -230,8 +244,10 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
         const int grid = want < (unsigned long long)shape.grid ? int(want) : shape.grid;
         rc = launch(ctx, ki, grid, &p, stream);
         if (rc != OMNI_OK) return rc;
+        if (grid > slots) slots = grid;
         ++launched;
     }
+    ctx->sq_slots = slots;
     // Alternate the sweep direction from call to call: the parameters and momentum touched last
     // are the ones still in L2 (loaded and stored with evict-last priority), so the next call
     // starts where this one ended and finds part of them there instead of in DRAM.
@@ -470,6 +486,8 @@ int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n
     if (rc != OMNI_OK) return rc;
     ctx->tally.weight_sum = wsum;
     ctx->tally.steps += 1;
+    rc = finalize_sqnorm(ctx, s);
+    if (rc != OMNI_OK) return rc;
     OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->host_cell, &ctx->ws->sqnorm, sizeof(double), cudaMemcpyDeviceToHost, s));
     OMNI_CUDA(ctx, cudaStreamSynchronize(s));
     if (grad_sqnorm) *grad_sqnorm = *ctx->host_cell;
@@ -776,11 +794,13 @@ int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream)
     if (!ctx || !out) return OMNI_ERR_NULL;
     if (ctx->ws) {
         cudaStream_t s = static_cast<cudaStream_t>(stream);
+        const int rc = finalize_sqnorm(ctx, s);
+        if (rc != OMNI_OK) return rc;
         OMNI_CUDA(ctx, cudaMemcpyAsync(ctx->host_cell, &ctx->ws->sqnorm, 2 * sizeof(double), cudaMemcpyDeviceToHost, s));
         OMNI_CUDA(ctx, cudaStreamSynchronize(s));
         ctx->tally.grad_sqnorm = ctx->host_cell[0];
         unsigned int words[2];
-        std::memcpy(words, &ctx->host_cell[1], sizeof words);   // ticket, status
+        std::memcpy(words, &ctx->host_cell[1], sizeof words);   // reserved, status
         if (words[1] != 0) {
             // a bounded device-side wait ran out in some earlier launch: report once and clear
             OMNI_CUDA(ctx, cudaMemsetAsync(&ctx->ws->status, 0, sizeof(unsigned int), s));

@@ -31,7 +31,15 @@ def _case(seed):
     alpha = float(rng.choice([1.0, 0.5, 0.25]))
     mode = int(rng.choice([B.BSP, B.BSP, B.ASP]))
     flags = int(rng.choice([0, 0, B.INPUT_IS_TIME]))
+    if rng.random() < 0.3:                           # the multiplicative reading of the global-batch rule
+        flags |= B.CONSERVE_MULTIPLICATIVE
     return rng, K, B_, b_min, b_max, deadband, alpha, mode, flags
+
+
+def _oracle_flags(flags):
+    """The oracle numbers its flags independently of the library."""
+    return ((O.FLAG_INPUT_IS_TIME if flags & B.INPUT_IS_TIME else 0)
+            | (O.FLAG_CONSERVE_MULTIPLICATIVE if flags & B.CONSERVE_MULTIPLICATIVE else 0))
 
 
 @pytest.mark.parametrize("seed", range(40))
@@ -40,7 +48,7 @@ def test_device_rebatch_matches_the_oracle_bit_for_bit(seed):
     device copy's batches equal the oracle's, and so do the weights it leaves for the step."""
     rng, K, B_, b_min, b_max, deadband, alpha, mode, flags = _case(1000 + seed)
     o = B.Omni(K, B_, b_min, b_max, deadband, alpha, mode, flags)
-    ref = O.Controller(K, B_, b_min, b_max, deadband, alpha, mode, flags)
+    ref = O.Controller(K, B_, b_min, b_max, deadband, alpha, mode, _oracle_flags(flags))
     assert list(ref.batches) == o.batches
     o.ctl_to_device()
     base = 8.0 ** rng.random(K)

@@ -69,8 +69,10 @@ def test_rebatch_bit_exact_against_oracle_random_traces(mode):
         db = float(rng.choice([0.0, 0.05, 0.1, 0.15]))
         alpha = float(rng.choice([1.0, 0.5, 0.3]))
         flags = int(rng.choice([0, B.INPUT_IS_TIME]))
-        lib = B.Omni(K, Bg, b_min, b_max, db, alpha, mode, flags)
-        ora = O.Controller(K, Bg, b_min, b_max, db, alpha, mode, flags)
+        mult = bool(rng.uniform() < 0.4)                 # the multiplicative reading of the global-batch rule
+        lib = B.Omni(K, Bg, b_min, b_max, db, alpha, mode, flags | (B.CONSERVE_MULTIPLICATIVE if mult else 0))
+        ora = O.Controller(K, Bg, b_min, b_max, db, alpha, mode,
+                           (O.FLAG_INPUT_IS_TIME if flags else 0) | (O.FLAG_CONSERVE_MULTIPLICATIVE if mult else 0))
         assert lib.batches == ora.batches.tolist()
         base = 8.0 ** rng.uniform(0, 1, K)
         for step in range(12):
@@ -105,6 +107,18 @@ def test_asp_report_bit_exact_against_oracle():
             assert a == b
             cur[k] = a
         assert lib.batches == ora.batches.tolist()
+
+
+def test_multiplicative_conservation_hand_cases():
+    import json
+
+    gold = json.loads((ROOT / "tests" / "golden" / "controller_cases.json").read_text())
+    for case in gold["multiplicative_cases"]:
+        o = B.Omni(case["K"], case["B"], case["b_min"], case["b_max"], case["deadband"], 1.0, B.BSP,
+                   B.CONSERVE_MULTIPLICATIVE)
+        assert o.batches == case["b0"]
+        for want in case["expect"]:
+            assert o.rebatch(case["throughput"])[0] == want, case["name"]
 
 
 def test_asp_report_hand_derived_sequences():
