@@ -32,6 +32,8 @@ sys.path.insert(0, str(ROOT))
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 HEADLINE = "resnet50_bf16"
+REPEATS = 5            # timed regions per configuration; the line reports their median and their best
+SCRUB_BYTES = 512 << 20  # written between steps by the cold-L2 legs (L2 holds 126 MB)
 METRIC = "params/sec, weighted aggregate+update (achieved HBM GB/s in roofline)"
 UNIT = "params/s"
 
@@ -40,8 +42,10 @@ UNIT = "params/s"
 # clocks
 # --------------------------------------------------------------------------------------------
 class ClockSampler:
-    """Reads SM clock and clock-event reasons of one GPU every 20 ms while the timed region runs."""
+    """Reads SM clock and clock-event reasons of one GPU every 2 ms, from the first warm-up step to
+    the end of the last timed repeat."""
 
+    PERIOD_S = 0.002
     REASONS = {
         0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
         0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting",
@@ -72,22 +76,23 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(self.PERIOD_S)
 
-    def __enter__(self):
-        if self._nv is not None:
+    def start(self):
+        if self._nv is not None and self._thread is None:
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
         return self
 
-    def __exit__(self, *a):
+    def stop(self):
         self._stop.set()
         if self._thread:
             self._thread.join()
 
     def summary(self):
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
-                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "period_ms": self.PERIOD_S * 1e3}
 
 
 def visible_index(local: int) -> int:
@@ -161,41 +166,88 @@ class BspJob:
             b, _ = o.rebatch(schedule[i % len(schedule)])
             o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
 
-    def timed(self, steps, warmup, schedule, sampler=None, barrier=None):
+    def timed(self, steps, warmup, schedule, sampler=None, barrier=None, repeats=REPEATS, reduce=None):
+        """``warmup`` untimed steps, then ``repeats`` timed regions of exactly ``steps`` steps, each
+        bracketed by a barrier + synchronize on both sides and timed with CUDA events on the
+        launching stream.  Returns (sorted ms per region -- after ``reduce``, the max over ranks --,
+        kernel launches per region)."""
         torch = self.torch
+        if sampler:
+            sampler.start()
         self.run(warmup, schedule)
-        torch.cuda.synchronize()
-        if barrier:
-            barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        l0 = self.omni.kernel_launches
-        torch.cuda.synchronize()
+        times, launches = [], 0
+        for _ in range(repeats):
+            torch.cuda.synchronize()
+            if barrier:
+                barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            l0 = self.omni.kernel_launches
+            e0.record()
+            self.run(steps, schedule)
+            e1.record()
+            torch.cuda.synchronize()
+            if barrier:
+                barrier()
+            ms = e0.elapsed_time(e1)
+            times.append(reduce(ms) if reduce else ms)
+            launches = self.omni.kernel_launches - l0
         if sampler:
-            sampler.__enter__()
-        e0.record()
-        self.run(steps, schedule)
-        e1.record()
+            sampler.stop()
+        return sorted(times), launches
+
+    def per_step(self, steps, schedule, between):
+        """Every step timed on its own (one event pair per step) with ``between()`` enqueued on the
+        same stream before it: what a step costs when it cannot find its predecessor's data in L2.
+        Returns the per-step times in ms."""
+        torch = self.torch
+        o, bs, cfg = self.omni, self.buckets, self.cfg
+        for i in range(3):
+            between()
+            b, _ = o.rebatch(schedule[i % len(schedule)])
+            o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
         torch.cuda.synchronize()
-        if sampler:
-            sampler.__exit__()
-        if barrier:
-            barrier()
-        return e0.elapsed_time(e1), self.omni.kernel_launches - l0
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps):
+            between()
+            b, _ = o.rebatch(schedule[i % len(schedule)])
+            ev[i][0].record()
+            o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(c) for a, c in ev]
 
 
-def bsp_line(job, ms, steps, launches, peak):
+def bsp_line(job, times, steps, launches, peak):
+    """``times``: sorted ms of the timed regions (each ``steps`` steps, ``launches`` kernels)."""
+    if not isinstance(times, (list, tuple)):
+        times = [times]
+    ms, best = statistics.median(times), min(times)
     per_launch_s = ms * 1e-3 / max(launches, 1)
     gbs = job.bytes_per_step * steps / max(launches, 1) / per_launch_s / 1e9
-    return {"params_per_s": job.cfg.P * steps / (ms * 1e-3), "ms_per_step": ms / steps, "achieved_gbs": gbs,
+    return {"params_per_s": job.cfg.P * steps / (ms * 1e-3), "ms_per_step": ms / steps,
+            "ms_per_step_best": best / steps, "repeats": len(times), "achieved_gbs": gbs,
             "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
             "bytes_per_param": job.bytes_per_step // job.cfg.P, "launches_per_step": launches / steps}
+
+
+def cold_line(job, per_step_ms, peak, what):
+    """Per-step times of a leg whose steps cannot reuse anything from L2."""
+    ms = statistics.median(per_step_ms)
+    gbs = job.bytes_per_step / (ms * 1e-3) / 1e9
+    return {"ms_per_step": ms, "ms_per_step_best": min(per_step_ms), "steps": len(per_step_ms), "achieved_gbs": gbs,
+            "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+            "params_per_s": job.cfg.P / (ms * 1e-3), "between_steps": what,
+            "timing": "one CUDA-event pair per step, median over the steps"}
 
 
 # --------------------------------------------------------------------------------------------
 # CPU oracle legs
 # --------------------------------------------------------------------------------------------
 def oracle_sample(name, n_max, torch, W):
-    """The single-threaded oracle on a prefix (at most n_max elements) of the configuration's first bucket."""
+    """The single-threaded oracle on a prefix (at most n_max elements) of the configuration's first
+    bucket, with the configuration's K, dtypes, optimiser constants and controller.  Returns
+    (elements, step function); one step is a re-batch + fused step (synchronous configurations)
+    or one arrival + report (the asynchronous one)."""
     from oracle import oracle as O
     import numpy as np
 
@@ -208,9 +260,20 @@ def oracle_sample(name, n_max, torch, W):
         t = torch.empty(n).normal_(0, 1e-3, generator=gen).to(gdt)
         g.append(t.view(torch.int16).numpy().view(np.uint16).copy() if gdt == torch.bfloat16 else t.numpy().copy())
     theta = torch.empty(n).normal_(0, cfg.param_std, generator=gen).numpy().copy()
+    base, sched = throughput_schedule(cfg, 64, W, torch)
+    if cfg.mode == "asp":
+        ctl = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, O.MODE_ASP)
+        u = torch.rand(4096, generator=gen, dtype=torch.float64).tolist()
+        b = [cfg.global_batch // cfg.K] * cfg.K
+
+        def step(i):
+            k = W.pick_worker(u[i % len(u)], [base[j] / b[j] for j in range(cfg.K)])
+            O.asp_apply_f32(g[k], b[k], cfg.global_batch, theta, None, cfg.lr, 0.0, 0.0)
+            b[k] = ctl.asp_report(k, b[k], base[k])
+
+        return n, step
     v = np.zeros(n, np.float32)
     ctl = O.Controller(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha)
-    base, sched = throughput_schedule(cfg, 64, W, torch)
 
     def step(i):
         b, _ = ctl.rebatch(sched[i % len(sched)])
@@ -219,8 +282,8 @@ def oracle_sample(name, n_max, torch, W):
     return n, step
 
 
-def cpu_baseline(name, target_s, torch, W):
-    n, step = oracle_sample(name, 4_000_000, torch, W)
+def cpu_baseline(name, target_s, torch, W, n_max=4_000_000):
+    n, step = oracle_sample(name, n_max, torch, W)
     step(0)
     t0 = time.perf_counter()
     step(1)
@@ -230,9 +293,11 @@ def cpu_baseline(name, target_s, torch, W):
     for i in range(reps):
         step(2 + i)
     dt = time.perf_counter() - t0
+    cfg = W.config(name)
+    unit = "arrivals" if cfg.mode == "asp" else "steps"
     return {"value": n * reps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{reps} steps over the first {n} elements of bucket 0 of {name} (K and dtypes as configured), "
-                      f"single thread, {dt:.1f} s",
+            "sample": f"{reps} {unit} over the first {n} elements of bucket 0 of {name} (K = {cfg.K}, {cfg.grad_dtype} "
+                      f"gradients, controller included), single thread, {dt:.1f} s",
             "host_cores_available": len(os.sched_getaffinity(0))}
 
 
@@ -320,8 +385,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="omni", choices=["omni", "reference"])
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--extras", default="all", choices=["all", "none", "asp", "ksweep"],
-                    help="which of the other configurations to time as well (not part of `value`)")
+    ap.add_argument("--extras", default="all", choices=["all", "none", "asp", "ksweep", "sharded"],
+                    help="which of the other configurations to time as well (not part of `value`); `sharded` "
+                         "(several ranks only) adds the parameter-range-sharded step: worker k's gradient lives "
+                         "on rank k mod N, every rank steps its own ranges over local and peer-mapped gradients")
+    ap.add_argument("--sharded-exchange", default="nccl", choices=["nccl", "ipc"],
+                    help="how the sharded leg returns the updated ranges: one NCCL all-gather per tensor (one "
+                         "rank per GPU), or device copies out of the peers' IPC-mapped buffers with gloo for the "
+                         "host-side protocol (also works with several ranks on one GPU)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -339,8 +410,11 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     B.lib()
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    ipc_mode = args.extras == "sharded" and args.sharded_exchange == "ipc"
+    if ipc_mode:
+        local %= torch.cuda.device_count()       # several ranks may share a GPU in this mode
     torch.cuda.set_device(local)
-    ranks = Ranks("nccl", torch.device("cuda", local))
+    ranks = Ranks("gloo", None) if ipc_mode else Ranks("nccl", torch.device("cuda", local))
     rank, world, dist = ranks.rank, ranks.world, ranks.dist
 
     def barrier():
@@ -354,10 +428,31 @@ def main():
     cfg = job.cfg
     _, sched = throughput_schedule(cfg, 256, W, torch)
     sampler = ClockSampler(visible_index(local))
-    ms, launches = job.timed(args.steps, args.warmup, sched, sampler, barrier)
-    ms = max_over_ranks(ms)
-    line_main = bsp_line(job, ms, args.steps, launches, peak)
+    times, launches = job.timed(args.steps, args.warmup, sched, sampler, barrier, REPEATS, max_over_ranks)
+    line_main = bsp_line(job, times, args.steps, launches, peak)
+    ms = statistics.median(times)
     grid, block = job.omni.query_launch(cfg.K, B.BF16)
+    n_buckets, bytes_per_step = len(job.buf.layout.buckets), job.bytes_per_step
+
+    # The same step when it cannot find its predecessor's theta and v in L2, every step timed on its
+    # own: (a) all K gradient buffers rewritten from a spare set between two steps, as the backward
+    # pass of a training loop would; (b) 512 MB written between two steps, which also leaves L2
+    # full of foreign dirty lines that the step has to push out.
+    fresh = cold = None
+    if rank == 0 and world == 1:
+        n_cold = max(20, min(args.steps, 200))
+        scrub = torch.empty(SCRUB_BYTES, dtype=torch.uint8, device=job.buf.theta.device)
+        spare = [g.clone() for g in job.buf.grads]
+
+        def rewrite_gradients():
+            for g, src in zip(job.buf.grads, spare):
+                g.copy_(src)
+
+        fresh = cold_line(job, job.per_step(n_cold, sched, rewrite_gradients), peak,
+                          "the K gradient buffers are rewritten by device copies from a spare set")
+        cold = cold_line(job, job.per_step(n_cold, sched, lambda: scrub.fill_(1)), peak,
+                         f"{SCRUB_BYTES >> 20} MB written to a scratch buffer (L2 flush)")
+        del spare, scrub
 
     # end to end: gradients arrive in pinned host memory, every step copies them in and reads the norm back
     e2e_steps = max(3, min(args.steps, 20))
@@ -385,33 +480,62 @@ def main():
         if args.extras == "ksweep":
             extras = run_k_sweep(torch, B, peak)
         else:
-            extras = run_extras(torch, W, B, peak, job, only_asp=args.extras == "asp")
+            extras = run_extras(torch, W, B, peak, job, only_asp=args.extras == "asp",
+                                with_cpu=not args.no_cpu_baseline)
+    if args.extras == "sharded" and world > 1:
+        del job
+        torch.cuda.empty_cache()
+        sh = run_sharded(torch, W, B, ranks, peak, max(3, min(args.steps, 200)), args.sharded_exchange)
+        if rank == 0:
+            extras["resnet50_bf16+sharded"] = sh
+        job = None
+    if fresh:
+        extras[HEADLINE + "+fresh_gradients"] = fresh
+        extras[HEADLINE + "+cold_l2"] = cold
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(HEADLINE, 12.0, torch, W)
 
-    traffic = recorded_traffic("bsp_tma_bf16_k16" if block == 288 else "bsp_fused_bf16_k16")
+    ring = block == 288
+    traffic = recorded_traffic("bsp_tma_bf16_k16" if ring else "bsp_fused_bf16_k16")
+    per_launch_s = ms * 1e-3 / max(launches, 1)
     if rank == 0:
         line = {
             "metric": METRIC, "value": world * line_main["params_per_s"], "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": line_main["ms_per_step"],
+            "ms_per_step_best": line_main["ms_per_step_best"], "repeats": REPEATS,
+            "ms_per_step_all_repeats": [t / args.steps for t in times],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": HEADLINE, "K": cfg.K, "params": cfg.P, "tensors": len(cfg.shapes),
-                       "buckets": len(job.buf.layout.buckets), "grad_dtype": "bf16", "master_dtype": "f32",
+                       "buckets": n_buckets, "grad_dtype": "bf16", "master_dtype": "f32",
                        "global_batch": cfg.global_batch, "lr": cfg.lr, "momentum": cfg.momentum,
-                       "rebatch": "every step", "l2": "inputs exceed L2 (1.23 GB touched per step)",
+                       "rebatch": "every step",
+                       "l2": "no flush in the headline region: a step touches 1.23 GB against 126 MB of L2, but "
+                             "back-to-back steps do find about 11 % of theta/v from their predecessor there; "
+                             "roofline.frac_fresh and roofline.frac_cold are the same step without that reuse",
+                       "timing": f"median of {REPEATS} regions of `steps` steps each",
                        "multi_gpu": "replicas only", "grid": grid, "block": block},
             "achieved_hbm_gbs": line_main["achieved_gbs"],
             "pct_of_nominal_8TBs": 100 * line_main["frac_of_nominal_8TBs"],
             "roofline": {"bound": "hbm", "achieved": line_main["achieved_gbs"], "peak": peak, "unit": "GB/s",
                          "frac": line_main["frac_of_measured"], "peak_source": f"of {peak_kind}",
-                         "kernel": "bsp_tma_kernel<bf16,16,tile 2048,2 stages>" if block == 288 else "bsp_fused_kernel<bf16,16>", "bytes_per_launch": job.bytes_per_step,
-                         "note": "algorithmic bytes; part of theta/v is re-used from L2 between launches, so DRAM traffic per launch is lower (see traffic) and the fraction can exceed 1",
+                         "kernel": "bsp_tma_kernel<bf16,16,tile 2048,2 stages>" if ring else "bsp_fused_kernel<bf16,16>",
+                         "bytes_per_launch": bytes_per_step,
+                         "note": "frac = algorithmic bytes over the mean launch time of back-to-back steps; there part "
+                                 "of theta/v comes from L2 (left by the previous step), so DRAM traffic per launch is "
+                                 "lower (traffic, dram_frac) and frac can exceed 1.  frac_fresh: every step timed alone "
+                                 "after all K gradient buffers were rewritten (a training loop's backward pass); "
+                                 "frac_cold: after 512 MB were written through L2.  The >= 80 % of nominal HBM claim "
+                                 "is to be read off frac_cold x peak / 8000 (pct_of_nominal_8TBs_cold).",
+                         "frac_fresh": fresh["frac_of_measured"] if fresh else None,
+                         "frac_cold": cold["frac_of_measured"] if cold else None,
+                         "pct_of_nominal_8TBs_fresh": 100 * fresh["frac_of_nominal_8TBs"] if fresh else None,
+                         "pct_of_nominal_8TBs_cold": 100 * cold["frac_of_nominal_8TBs"] if cold else None,
                          "traffic": traffic,
-                         # what DRAM actually served per second: the ncu traffic per launch over this run's launch time
-                         "dram_gbs": (traffic / (ms * 1e-3 / max(launches, 1)) / 1e9) if traffic else None,
-                         "dram_frac": (traffic / (ms * 1e-3 / max(launches, 1)) / 1e9 / peak) if traffic else None},
+                         # what DRAM served per second: the ncu traffic per launch over this run's launch time
+                         "dram_gbs": (traffic / per_launch_s / 1e9) if traffic else None,
+                         "dram_frac": (traffic / per_launch_s / 1e9 / peak) if traffic else None},
             "e2e": {"value": world * cfg.P * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": 8, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": launches,
@@ -421,6 +545,87 @@ def main():
         }
         print(json.dumps(line))
     ranks.close()
+
+
+def run_sharded(torch, W, B, ranks, peak, steps, how):
+    """The headline step sharded by parameter range over the ranks (Algorithm 1's AllReduce as a
+    reduce-scatter): worker k's gradient buffer lives on rank k mod N, every rank holds a replica
+    of theta and v, maps the other ranks' gradient buffers through CUDA IPC, runs the fused step
+    on the ranges it owns -- reading N-th of the gradients locally and the rest from the peers'
+    memory -- and the updated ranges travel back by one all-gather per tensor (NCCL) or by device
+    copies out of the peers' mapped replicas (`ipc`).  Time = max over ranks of the CUDA-event
+    time of `steps` such steps; the result is checked against the unsharded step on rank 0."""
+    from paper_2503_17469_b200 import sharded as S
+
+    dist, world, rank = ranks.dist, ranks.world, ranks.rank
+    cfg = W.config(HEADLINE)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    buf = W.make_buffers(cfg, dev)                      # same seed on every rank: identical replicas
+    lay = buf.layout
+    mine = [k for k in range(cfg.K) if k % world == rank]
+    own = [buf.grads[k] for k in mine]
+    reference = None
+    if rank == 0:                                       # the unsharded result, for the check at the end
+        ref_theta, ref_v = buf.theta.clone(), buf.v.clone()
+        reference = (ref_theta, ref_v, B.BucketSet.from_flat(lay, ref_theta, buf.grads, ref_v))
+    else:
+        buf.grads = [g if k in mine else None for k, g in enumerate(buf.grads)]   # free the other workers' gradients
+    torch.cuda.empty_cache()
+    torch.cuda.synchronize()
+    views = S.map_peers(own + [buf.theta, buf.v], dist)
+    for r in range(world):                              # first touch of a peer's memory enables peer access
+        if r != rank:
+            torch.empty(1, dtype=views[r][0].dtype, device=dev).copy_(views[r][0][:1])
+    flat_g = [views[k % world][[kk for kk in range(cfg.K) if kk % world == k % world].index(k)] for k in range(cfg.K)]
+    sl = [slice(b.start, b.start + b.n) for b in lay.buckets]
+    theta_b, v_b = [buf.theta[x] for x in sl], [buf.v[x] for x in sl]
+    grads_b = [[g[x] for g in flat_g] for x in sl]
+    state_views = [[t[x] for t in vw[-2:] for x in sl] for vw in views]      # every rank's theta and v, by bucket
+    shard = S.shard_buckets(theta_b, grads_b, v_b, None, world, rank)
+    o = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.BSP)
+    _, sched = throughput_schedule(cfg, 64, W, torch)
+
+    def step(i):
+        b, _ = o.rebatch(sched[i % len(sched)])
+        o.aggregate_bsp(shard, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+        if how == "nccl":
+            S.all_gather_ranges(theta_b + v_b, world, rank, dist)
+        else:
+            torch.cuda.synchronize()
+            dist.barrier()                              # every owner has updated its ranges
+            S.pull_ranges(theta_b + v_b, state_views, world, rank)
+            torch.cuda.synchronize()
+            dist.barrier()                              # nobody steps again before everyone has pulled
+        return b
+
+    batches = [step(i) for i in range(3)]
+    torch.cuda.synchronize()
+    ranks.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    batches += [step(3 + i) for i in range(steps)]
+    e1.record()
+    torch.cuda.synchronize()
+    ranks.barrier()
+    ms = ranks.max_over_ranks(e0.elapsed_time(e1))
+    ok = None
+    if rank == 0:
+        ref_theta, ref_v, ref_bs = reference
+        ro = B.Omni(cfg.K, cfg.global_batch, cfg.b_min, cfg.b_max, cfg.deadband, cfg.ewma_alpha, B.BSP)
+        for b in batches:
+            ro.aggregate_bsp(ref_bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+        torch.cuda.synchronize()
+        ok = bool(torch.equal(ref_theta, buf.theta) and torch.equal(ref_v, buf.v))
+    del views, flat_g, grads_b, state_views, shard
+    ranks.barrier()
+    nccl_bytes = 8 * cfg.P * (world - 1) / world        # theta + v ranges a rank receives per step
+    return {"ms_per_step": ms / steps, "params_per_s": cfg.P * steps / (ms * 1e-3), "ranks": world, "exchange": how,
+            "steps": steps, "matches_unsharded_step_bit_for_bit": ok,
+            "bytes_per_rank_per_step": {"gradients_local": cfg.P // world * 2 * len(mine),
+                                        "gradients_from_peers": cfg.P // world * 2 * (cfg.K - len(mine)),
+                                        "theta_v_read_write": cfg.P // world * 16, "exchange_received": nccl_bytes},
+            "note": "whole-job rate of ONE model updated by all ranks together (strong scaling of the step), "
+                    "unlike `value`, which counts independent replicas"}
 
 
 def run_k_sweep(torch, B, peak, P=25_557_032, steps=200):
@@ -461,11 +666,45 @@ def run_k_sweep(torch, B, peak, P=25_557_032, steps=200):
     return out
 
 
-def run_extras(torch, W, B, peak, headline_job, only_asp=False):
-    """The other configurations, each timed with CUDA events after warm-up (not part of `value`)."""
+def timed_replays(torch, graph, replays, before=None, repeats=REPEATS):
+    """Sorted ms of ``repeats`` regions of ``replays`` replays of a CUDA graph."""
+    times = []
+    for _ in range(repeats):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(replays):
+            if before:
+                before(i)
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return sorted(times)
+
+
+def timed_calls(torch, fn, first, count, repeats=REPEATS):
+    """Sorted ms of ``repeats`` regions in which ``fn(i0, count)`` enqueues ``count`` calls."""
+    times = []
+    for r in range(repeats):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn(first + r * count, count)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    return sorted(times)
+
+
+def run_extras(torch, W, B, peak, headline_job, only_asp=False, with_cpu=True):
+    """The other configurations, each timed with CUDA events after warm-up (not part of `value`):
+    median and best of REPEATS regions, the cold-L2 figure of the synchronous ones, and the CPU
+    oracle on a prefix of each configuration."""
     out = {}
     del headline_job
     torch.cuda.empty_cache()
+    scrub = torch.empty(SCRUB_BYTES, dtype=torch.uint8, device="cuda")
     for name, steps, lp, flags in (("resnet50_bf16", 500, True, 0),
                                    ("resnet50_bf16", 500, False, B.NO_BULK_COPY),
                                    ("resnet50_f32", 500, False, 0), ("resnet50_f32", 500, False, B.NO_BULK_COPY),
@@ -474,9 +713,14 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
             break
         job = BspJob(name, torch, W, B, with_lp=lp, flags=flags)
         _, sched = throughput_schedule(job.cfg, 64, W, torch)
-        ms, launches = job.timed(steps, 5, sched)
+        times, launches = job.timed(steps, 5, sched)
         key = name + ("+lp_copy" if lp else "") + ("+register_kernels" if flags else "")
-        out[key] = bsp_line(job, ms, steps, launches, peak)
+        out[key] = bsp_line(job, times, steps, launches, peak)
+        if name != "tiny":
+            out[key]["cold_l2"] = cold_line(job, job.per_step(40 if name != "vgg16" else 10, sched, lambda: scrub.fill_(1)),
+                                            peak, f"{SCRUB_BYTES >> 20} MB written to a scratch buffer (L2 flush)")
+        if with_cpu and not lp and not flags and name != HEADLINE:
+            out[key]["cpu_baseline"] = cpu_baseline(name, 2.5, torch, W, n_max=1_000_000)
         if name == "tiny":
             out[key]["note"] = "33.6 MB working set: L2-resident and launch-bound, not an HBM figure"
             # the same steps with the launches captured once in a CUDA graph (fixed batches)
@@ -491,15 +735,7 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
                     job.omni.aggregate_bsp(job.buckets, b, job.cfg.lr, job.cfg.momentum)
             for _ in range(3):
                 graph.replay()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(40):
-                graph.replay()
-            e1.record()
-            torch.cuda.synchronize()
-            gms = e0.elapsed_time(e1)
-            out[key + "+cuda_graph"] = bsp_line(job, gms, 2000, 2000, peak)
+            out[key + "+cuda_graph"] = bsp_line(job, timed_replays(torch, graph, 40), 2000, 2000, peak)
             out[key + "+cuda_graph"]["note"] = "50 steps per graph, fixed batches; L2-resident"
             del graph
             # whole steps (device-side re-batch + fused step with device-resident weights) in a graph
@@ -516,14 +752,10 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
                     job.omni.aggregate_bsp_device_batches(job.buckets, job.cfg.lr, job.cfg.momentum)
             for _ in range(3):
                 graph.replay()
-            torch.cuda.synchronize()
-            e0.record()
-            for i in range(40):
-                measured.copy_(torch.tensor(sched[i % len(sched)], dtype=torch.float64), non_blocking=False)
-                graph.replay()
-            e1.record()
-            torch.cuda.synchronize()
-            out[key + "+device_controller_graph"] = bsp_line(job, e0.elapsed_time(e1), 2000, 2000, peak)
+            host_sched = [torch.tensor(m, dtype=torch.float64) for m in sched]
+            new_measurements = lambda i: measured.copy_(host_sched[i % len(host_sched)], non_blocking=False)
+            out[key + "+device_controller_graph"] = bsp_line(job, timed_replays(torch, graph, 40, new_measurements),
+                                                             2000, 2000, peak)
             out[key + "+device_controller_graph"]["launches_per_step"] = 2.0
             out[key + "+device_controller_graph"]["note"] = ("50 x (one-warp re-batch kernel + fused step reading its "
                                                              "weights from device memory) per graph, new measurements "
@@ -545,13 +777,8 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
                 job.omni.aggregate_bsp_device_batches(job.buckets, job.cfg.lr, job.cfg.momentum)
 
         dev_run(5)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        dev_run(500)
-        e1.record()
-        torch.cuda.synchronize()
-        out["resnet50_bf16+device_controller"] = bsp_line(job, e0.elapsed_time(e1), 500, 500, peak)
+        out["resnet50_bf16+device_controller"] = bsp_line(job, timed_calls(torch, lambda i0, n: dev_run(n), 0, 500),
+                                                          500, 500, peak)
         out["resnet50_bf16+device_controller"]["launches_per_step"] = 2.0
         out["resnet50_bf16+device_controller"]["note"] = "re-batch kernel (1 warp) + fused step per step; GB/s counts the step's bytes over the time of both"
         job.omni.ctl_from_device()
@@ -564,9 +791,28 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
     bs = B.BucketSet.from_flat(buf.layout, buf.theta, buf.grads)
     gen = torch.Generator().manual_seed(cfg.seed)
     T = W.draw_throughputs(cfg.K, gen, cfg.ratio)
-    u = torch.rand(cfg.steps + 64, generator=gen, dtype=torch.float64).tolist()
+    u = torch.rand(64 + (REPEATS + 1) * cfg.steps, generator=gen, dtype=torch.float64).tolist()
     b = [cfg.global_batch // cfg.K] * cfg.K
     last = [0] * cfg.K
+
+    def asp_line(times, n_arr, bpp, traffic_key=None, note=None):
+        """Asynchronous legs: theta (102 MB) and most of what an arrival touches stay in the 126 MB
+        L2 from one arrival to the next, so the algorithmic rate is NOT an HBM figure; it is
+        printed beside the copy peak only for scale, and the DRAM-side rate (ncu traffic per
+        arrival over this run's time) and the cold-L2 leg are the HBM figures."""
+        ms = statistics.median(times)
+        gbs = bpp * cfg.P * n_arr / (ms * 1e-3) / 1e9
+        traffic = recorded_traffic(traffic_key) if traffic_key else None
+        per_arrival_s = ms * 1e-3 / n_arr
+        line = {"params_per_s": cfg.P * n_arr / (ms * 1e-3), "ms_per_arrival": ms / n_arr,
+                "ms_per_arrival_best": min(times) / n_arr, "repeats": len(times), "bytes_per_param": bpp,
+                "algorithmic_gbs": gbs, "algorithmic_vs_copy_peak": gbs / peak,
+                "bound": "L2 + launch (theta stays in L2 between arrivals; not an HBM roofline figure)",
+                "traffic": traffic, "dram_gbs": traffic / per_arrival_s / 1e9 if traffic else None,
+                "dram_frac": traffic / per_arrival_s / 1e9 / peak if traffic else None}
+        if note:
+            line["note"] = note
+        return line
 
     def arrivals(i0, n):
         for i in range(i0, i0 + n):
@@ -577,20 +823,30 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
 
     arrivals(0, 50)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     l0 = o.kernel_launches
-    e0.record()
-    arrivals(50, cfg.steps)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
+    times = timed_calls(torch, arrivals, 50, cfg.steps)
     st = o.stats()
-    gbs = cfg.bytes_per_param() * cfg.P * cfg.steps / (ms * 1e-3) / 1e9
-    out["resnet50_asp"] = {"params_per_s": cfg.P * cfg.steps / (ms * 1e-3), "ms_per_arrival": ms / cfg.steps,
-                           "achieved_gbs": gbs, "frac_of_measured": gbs / peak,
-                           "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_param": cfg.bytes_per_param(),
-                           "launches_per_arrival": (o.kernel_launches - l0) / cfg.steps, "tau_max": st.tau_max,
-                           "tau_hist_0_31_overflow": st.tau_hist}
+    out["resnet50_asp"] = asp_line(times, cfg.steps, cfg.bytes_per_param(), "asp_tma_f32_single_arrival")
+    out["resnet50_asp"].update({"launches_per_arrival": (o.kernel_launches - l0) / (REPEATS * cfg.steps),
+                                "tau_max": st.tau_max, "tau_hist_0_31_overflow": st.tau_hist})
+    # one arrival when theta is not in L2: 512 MB written between two arrivals, each timed on its own
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(40)]
+    i_next = 50 + REPEATS * cfg.steps
+    for j, (a, c) in enumerate(ev):
+        scrub.fill_(1)
+        k = W.pick_worker(u[i_next + j], [T[q] / b[q] for q in range(cfg.K)])
+        a.record()
+        o.apply_asp(bs, k, b[k], 0, cfg.lr)
+        c.record()
+    torch.cuda.synchronize()
+    ms_cold = statistics.median(a.elapsed_time(c) for a, c in ev)
+    gbs_cold = cfg.bytes_per_param() * cfg.P / (ms_cold * 1e-3) / 1e9
+    out["resnet50_asp"]["cold_l2"] = {"ms_per_arrival": ms_cold, "achieved_gbs": gbs_cold, "bound": "hbm",
+                                      "frac_of_measured": gbs_cold / peak, "frac_of_nominal_8TBs": gbs_cold / NOMINAL_HBM_GBS,
+                                      "between_arrivals": f"{SCRUB_BYTES >> 20} MB written to a scratch buffer (L2 flush)",
+                                      "timing": "one CUDA-event pair per arrival, median of 40"}
+    if with_cpu:
+        out["resnet50_asp"]["cpu_baseline"] = cpu_baseline("resnet50_asp", 2.5, torch, W, n_max=1_000_000)
     # Algorithm 2 taken literally on the same stream: the arriving worker's local step overwrites the server
     # copy (push), then the worker reads the new parameters back into its snapshot (pull)
     snaps = [torch.empty_like(buf.theta) for _ in range(cfg.K)]
@@ -598,8 +854,6 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
     snap_views = [[sn[bk.start:bk.start + bk.n] for bk in buf.layout.buckets] for sn in snaps]
     for k in range(cfg.K):
         o3.asp_pull(bs, snap_views[k])
-    b = [cfg.global_batch // cfg.K] * cfg.K
-    last = [0] * cfg.K
 
     def literal(i0, n):
         for i in range(i0, i0 + n):
@@ -619,23 +873,14 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
     for key, fn, bpp, note in (
             ("resnet50_asp_push_overwrite+pull", literal, 20,
              "per arrival: push (read snapshot + gradient, write theta: 12 B/param) + pull (device copies theta -> "
-             "snapshot: 8 B/param)"),
+             "snapshot: 8 B/param); the K snapshots (1.6 GB) do not fit L2, so this leg is mostly DRAM traffic"),
             ("resnet50_asp_push_pull_fused", fused, 16,
-             "per arrival: one pass reads snapshot + gradient and writes theta and the snapshot")):
+             "per arrival: one pass reads snapshot + gradient and writes theta and the snapshot; mostly DRAM traffic")):
         b[:] = [cfg.global_batch // cfg.K] * cfg.K
         last[:] = [0] * cfg.K
         fn(0, 50)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        fn(50, cfg.steps)
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        gbs = bpp * cfg.P * cfg.steps / (ms * 1e-3) / 1e9
-        out[key] = {"params_per_s": cfg.P * cfg.steps / (ms * 1e-3), "ms_per_arrival": ms / cfg.steps,
-                    "achieved_gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-                    "bytes_per_param": bpp, "note": note}
+        out[key] = asp_line(timed_calls(torch, fn, 50, cfg.steps), cfg.steps, bpp, note=note)
+        out[key]["bound"] = "hbm for the snapshot and gradient (read once per arrival), L2 for part of theta"
     del snaps, snap_views, o3
     # the same stream with arrivals queued four at a time and applied in one pass each
     m = 4
@@ -655,22 +900,11 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False):
                 b[k] = o2.asp_report(k, bu, T[k])
 
     batched(0, 48)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n_arr = cfg.steps // m * m
     l0 = o2.kernel_launches
-    e0.record()
-    batched(48, n_arr)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    bpp = (4 * m + 8) / m
-    gbs = bpp * cfg.P * n_arr / (ms * 1e-3) / 1e9
-    out["resnet50_asp_batched4"] = {"params_per_s": cfg.P * n_arr / (ms * 1e-3), "ms_per_arrival": ms / n_arr,
-                                    "achieved_gbs": gbs, "frac_of_measured": gbs / peak,
-                                    "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "bytes_per_param": bpp,
-                                    "launches_per_arrival": (o2.kernel_launches - l0) / n_arr,
-                                    "note": "4 queued arrivals per pass: 6 B/param/arrival instead of 12"}
+    out["resnet50_asp_batched4"] = asp_line(timed_calls(torch, batched, 48, n_arr), n_arr, (4 * m + 8) / m,
+                                            note="4 queued arrivals per pass: 6 B/param/arrival instead of 12")
+    out["resnet50_asp_batched4"]["launches_per_arrival"] = (o2.kernel_launches - l0) / (REPEATS * n_arr)
     return out
 
 

@@ -44,6 +44,24 @@ template <typename G> KernelInfo bulk_for(int K)
     return {};
 }
 
+// the same kernel in the shape for short launches (the very same instantiation where the shapes agree)
+template <typename G, int K> KernelInfo bulk_short_info()
+{
+    constexpr TmaShape sh = tma_short_shape<G>(K);
+    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps>),
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_ring_bytes(sh, K, int(sizeof(G))), true};
+}
+
+template <typename G> KernelInfo bulk_short_for(int K)
+{
+    switch (K) {
+#define OMNI_CASE(k) case k: return bulk_short_info<G, k>();
+        OMNI_FOR_EACH_K(OMNI_CASE)
+#undef OMNI_CASE
+    }
+    return {};
+}
+
 template <typename G, int M> KernelInfo bulk_seq_info()
 {
     constexpr TmaShape sh = tma_seq_shape<G>(M);
@@ -76,6 +94,11 @@ KernelInfo bulk_overwrite_kernel(int dtype)
 }
 
 KernelInfo bulk_kernel(int dtype, int K) { return dtype == OMNI_BF16 ? bulk_for<__nv_bfloat16>(K) : bulk_for<float>(K); }
+KernelInfo bulk_short_kernel(int dtype, int K)
+{
+    return dtype == OMNI_BF16 ? bulk_short_for<__nv_bfloat16>(K) : bulk_short_for<float>(K);
+}
+int short_launch_tiles_per_cta() { return kShortLaunchTilesPerCta; }
 KernelInfo bulk_seq_kernel(int dtype, int M) { return dtype == OMNI_BF16 ? bulk_seq_for<__nv_bfloat16>(M) : bulk_seq_for<float>(M); }
 
 int launch_sqnorm_finalize(void *workspace, int slots, double *out, void *stream)

@@ -39,6 +39,11 @@ KernelInfo overwrite_kernel(int dtype, bool wide);
 // asynchronous apply of M queued arrivals (M = 1: a single arrival; M <= OMNI_MAX_ASP_BATCH).
 KernelInfo bulk_kernel(int dtype, int K);
 KernelInfo bulk_seq_kernel(int dtype, int M);
+// The synchronous ring kernel in its shape for short launches (larger tiles, two stages; the same
+// kernel as bulk_kernel where no such shape fits), chosen when the regular shape would give a CTA
+// at most short_launch_tiles_per_cta() tiles and the larger tiles still number one per SM or more.
+KernelInfo bulk_short_kernel(int dtype, int K);
+int short_launch_tiles_per_cta();
 // The synchronous ring kernel that reads its K weights from device memory (BspParams::lam_dev),
 // where the device-side controller leaves them (device_controller.cu).
 KernelInfo bulk_devlam_kernel(int dtype, int K);

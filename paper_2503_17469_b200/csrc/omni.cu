@@ -32,6 +32,7 @@ struct omni_ctx {
     omni::DeviceCtl dctl_stage{};    // host staging for its uploads and downloads
     omni::LaunchShape bsp_shape[2][2][OMNI_MAX_K + 1];  // [dtype][wide][K]
     omni::LaunchShape bulk_shape[2][OMNI_MAX_K + 1];    // [dtype][K], bulk-copy ring kernel
+    omni::LaunchShape bulk_short_shape[2][OMNI_MAX_K + 1];  // [dtype][K], the same in its shape for short launches
     omni::LaunchShape bulk_seq_shape[2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][M]
     omni::LaunchShape bulk_devlam_shape[2][OMNI_MAX_K + 1];       // [dtype][K], ring kernel with device-resident weights
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
@@ -208,10 +209,26 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
     const int K = ctx->ctl.K();
     const bool bulk = lam_dev || use_bulk(ctx, dtype, K);
     const bool wide = all_aligned32(buckets, n_buckets, 0, K);
-    const KernelInfo ki = lam_dev ? bulk_devlam_kernel(dtype, K) : bulk ? bulk_kernel(dtype, K) : bsp_kernel(dtype, K, wide);
-    LaunchShape &shape = lam_dev ? ctx->bulk_devlam_shape[dtype][K]
-                         : bulk  ? ctx->bulk_shape[dtype][K]
-                                 : ctx->bsp_shape[dtype][wide][K];
+    KernelInfo ki = lam_dev ? bulk_devlam_kernel(dtype, K) : bulk ? bulk_kernel(dtype, K) : bsp_kernel(dtype, K, wide);
+    LaunchShape *shape_slot = lam_dev ? &ctx->bulk_devlam_shape[dtype][K]
+                              : bulk  ? &ctx->bulk_shape[dtype][K]
+                                      : &ctx->bsp_shape[dtype][wide][K];
+    if (bulk && !lam_dev) {
+        // a launch of a few rounds per CTA takes the short-launch shape, as long as that still
+        // gives every SM a tile
+        const KernelInfo ks = bulk_short_kernel(dtype, K);
+        unsigned long long regular_tiles = 0, short_tiles = 0;
+        for (int i = 0; i < n_buckets; ++i) {
+            regular_tiles += (buckets[i].n + ki.tile - 1) / ki.tile;
+            short_tiles += (buckets[i].n + ks.tile - 1) / ks.tile;
+        }
+        const unsigned long long sms = (unsigned long long)ctx->sm_count;
+        if (ks.fn != ki.fn && regular_tiles <= (unsigned long long)short_launch_tiles_per_cta() * sms && short_tiles >= sms) {
+            ki = ks;
+            shape_slot = &ctx->bulk_short_shape[dtype][K];
+        }
+    }
+    LaunchShape &shape = *shape_slot;
     int rc = shape_for(ctx, ki, shape);
     if (rc != OMNI_OK) return rc;
     const unsigned long long tile = ki.tile;

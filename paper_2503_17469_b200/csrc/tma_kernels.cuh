@@ -111,6 +111,29 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
     if (stages > 8) stages = 8;
     return {tile, stages, 8};
 }
+// Short launches.  A launch that gives every CTA only a handful of tiles never reaches the ring's
+// steady state: its time is a few rounds of "fill a stage, consume it", and what counts is how
+// much each round moves.  Where two stages of twice the regular tile still fit in shared memory
+// (float K = 4; bfloat16 K = 7, 8 -- smaller K already use 4096-element tiles, larger K do not
+// fit), that shape is used for such launches: on the cache-resident 2^20-parameter K = 4 model,
+// captured in a CUDA graph, 4096 x 2 runs a step in 4.40 us against 4.85 us for 2048 x 3 (and
+// 4.55 us for 2048 x 4, 5.2-5.4 us for 2048 x 2 and 1536 x 4; tiles of 1024 and 512 elements, which
+// balance the last wave better, were slower still: 8.0 and 11.4 us against 6.7 us before the norm's
+// final sum left the kernel).  The window is narrow: with 2^19 parameters (fewer large tiles than
+// SMs) the two shapes tie at 3.1 us, with 2^18 the regular one wins (2.4 vs 2.9 us), and from 2^21
+// parameters on (7 regular tiles per CTA) the regular shape's third stage wins again (6.7 vs
+// 7.1 us, 13.3 vs 13.7, 27.5 vs 28.4).  So the short shape is chosen when the regular shape
+// would give a CTA at most kShortLaunchTilesPerCta tiles and the large tiles still number at
+// least one per SM.
+constexpr int kShortLaunchTilesPerCta = 4;
+template <typename G> __host__ __device__ constexpr TmaShape tma_short_shape(int K)
+{
+    const TmaShape s = tma_shape<G>(K);
+    const int per_elem = K * int(sizeof(G)) + 8;
+    if (s.tile < 4096 && 2 * (2 * s.tile) * per_elem <= 200 * 1024) return {2 * s.tile, 2, s.consumer_warps};
+    return s;
+}
+
 // The asynchronous apply of M queued arrivals uses the same geometry with M streams, except for
 // the shortest queues: with most of theta coming from L2 (see the alternating sweeps in omni.cu)
 // they are no longer DRAM-bound, and a deeper ring with sixteen consumer warps gains 2-6 %

@@ -118,3 +118,29 @@ def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
     sq_o = O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 0.0)
     assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
     assert np.array_equal(to_np(theta.t), th_o)
+
+
+@pytest.mark.parametrize("kind,K", [("f32", 4), ("bf16", 7), ("bf16", 8)])
+def test_short_launches_take_larger_tiles_with_the_same_bits(kind, K):
+    """Launches of a few tiles per CTA run the ring in its short-launch shape (two stages of
+    4096-element tiles where they fit: float K = 4, bfloat16 K = 7 and 8).  Sizes inside that
+    window (a ragged tail, several buckets) and just outside it on both sides give the oracle's
+    bits either way."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for sizes in ([sms * 4096 + 77], [sms * 2048 * 4 - 5], [sms * 2048 + 3], [5 * sms * 2048 + 4099],
+                  [300_001, 77, 450_003, 4096]):
+        bufs = [_make(K, n, kind, 4100 * K + n % 983, lp=True) for n in sizes]
+        b = _random_batches(K, 32, K + sizes[0])
+        o = B.Omni(K, 32 * K, 1, 32 * K, 0.1, flags=B.BULK_COPY)
+        bs = B.BucketSet([x[0].t for x in bufs], [[g.t for g in x[2]] for x in bufs], [x[1].t for x in bufs],
+                         [x[3].t for x in bufs])
+        ora = [(to_np(x[0].t), to_np(x[1].t), np.zeros(n, np.uint16), [to_np(g.t) for g in x[2]]) for x, n in zip(bufs, sizes)]
+        for _ in range(2):
+            o.aggregate_bsp(bs, b, 0.1, 0.9, 5e-4)
+            sq_o = sum(O.bsp_step_f32(g_np, b, th_o, v_o, 0.1, 0.9, 5e-4, theta_lp=lp_o) for th_o, v_o, lp_o, g_np in ora)
+            assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+        for (theta, v, grads, plp), (th_o, v_o, lp_o, _) in zip(bufs, ora):
+            assert np.array_equal(to_np(theta.t), th_o) and np.array_equal(to_np(v.t), v_o), (K, sizes)
+            assert np.array_equal(to_np(plp.t), lp_o)
+            for buf in (theta, v, plp, *grads):
+                assert buf.intact(), "guard band overwritten"
