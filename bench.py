@@ -301,6 +301,14 @@ def cpu_baseline(name, target_s, torch, W, n_max=4_000_000):
             "host_cores_available": len(os.sched_getaffinity(0))}
 
 
+def headline_config(cfg, n_buckets):
+    """`config` of the JSON line: the workload, identical in both arms."""
+    return {"workload": HEADLINE, "K": cfg.K, "params": cfg.P, "tensors": len(cfg.shapes), "buckets": n_buckets,
+            "grad_dtype": "bf16", "master_dtype": "f32", "global_batch": cfg.global_batch, "lr": cfg.lr,
+            "momentum": cfg.momentum, "rebatch": "every step", "multi_gpu": "replicas only",
+            "l2": "inputs larger than L2 (1.23 GB touched per step, 126 MB of L2), no flush between the timed steps"}
+
+
 def reference_arm(args, torch, W):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -326,9 +334,9 @@ def reference_arm(args, torch, W):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": HEADLINE, "K": cfg.K, "params": cfg.P, "grad_dtype": cfg.grad_dtype,
-                       "global_batch": cfg.global_batch, "sample_elements": n},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "config": headline_config(cfg, len(cfg.layout().buckets)),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                             "sample_elements": n},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -507,15 +515,11 @@ def main():
             "ms_per_step_best": line_main["ms_per_step_best"], "repeats": REPEATS,
             "ms_per_step_all_repeats": [t / args.steps for t in times],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": HEADLINE, "K": cfg.K, "params": cfg.P, "tensors": len(cfg.shapes),
-                       "buckets": n_buckets, "grad_dtype": "bf16", "master_dtype": "f32",
-                       "global_batch": cfg.global_batch, "lr": cfg.lr, "momentum": cfg.momentum,
-                       "rebatch": "every step",
+            "config": headline_config(cfg, n_buckets),
+            "launch": {"grid": grid, "block": block, "timing": f"median of {REPEATS} regions of `steps` steps each",
                        "l2": "no flush in the headline region: a step touches 1.23 GB against 126 MB of L2, but "
                              "back-to-back steps do find about 11 % of theta/v from their predecessor there; "
-                             "roofline.frac_fresh and roofline.frac_cold are the same step without that reuse",
-                       "timing": f"median of {REPEATS} regions of `steps` steps each",
-                       "multi_gpu": "replicas only", "grid": grid, "block": block},
+                             "roofline.frac_fresh and roofline.frac_cold are the same step without that reuse"},
             "achieved_hbm_gbs": line_main["achieved_gbs"],
             "pct_of_nominal_8TBs": 100 * line_main["frac_of_nominal_8TBs"],
             "roofline": {"bound": "hbm", "achieved": line_main["achieved_gbs"], "peak": peak, "unit": "GB/s",

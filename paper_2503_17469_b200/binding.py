@@ -272,9 +272,13 @@ class Omni:
     # ---- device path ------------------------------------------------------------------------
     @staticmethod
     def _stream(stream) -> C.c_void_p:
+        """The raw cudaStream_t of ``stream`` (a torch stream), or of torch's current stream."""
         if stream is None:
             import torch
 
+            raw = getattr(torch._C, "_cuda_getCurrentRawStream", None)     # no Stream object built: the call sits
+            if raw is not None:                                            # on the path of every step
+                return C.c_void_p(raw(torch.cuda.current_device()))
             stream = torch.cuda.current_stream()
         return C.c_void_p(stream.cuda_stream)
 

@@ -262,6 +262,52 @@ def test_steps_replayed_from_a_cuda_graph():
     assert abs(o.stats().grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
 
 
+def test_ordinary_kernels_between_steps_see_finished_steps():
+    """The ring kernels signal early that dependents may launch; a kernel enqueued after a step in
+    the ordinary way (here: torch copies, eagerly and inside a captured graph) must still see the
+    step's finished theta and v, and a step that follows such a kernel must see its writes (the
+    gradient is rewritten between the steps)."""
+    K, n = 3, 5 * 8192 + 11
+    theta, v, grads, _ = _make(K, n, "f32", 654)
+    alt = [g.t.clone().mul_(-0.5) for g in grads]            # a second set of gradients to switch to
+    first = [g.t.clone() for g in grads]
+    o = B.Omni(K, 48, 1, 48, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    b = [5, 16, 27]
+    snaps = [torch.empty(n, device=DEV) for _ in range(4)]
+
+    def sequence():
+        for i in range(4):
+            src = first if i % 2 == 0 else alt
+            for g, s_ in zip(grads, src):
+                g.t.copy_(s_)                                    # ordinary kernels before the step ...
+            o.aggregate_bsp(bs, b, 0.1, 0.9)
+            snaps[i].copy_(theta.t)                              # ... and right after it
+
+    th_o, v_o = to_np(theta.t), to_np(v.t)
+    g_sets = [[to_np(x) for x in first], [to_np(x) for x in alt]]
+    want = []
+    for rep in range(3):                                         # one eager pass, two graph replays
+        for i in range(4):
+            O.bsp_step_f32(g_sets[i % 2], b, th_o, v_o, 0.1, 0.9, 0.0)
+            want.append(th_o.copy())
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        sequence()
+    side.synchronize()
+    for i in range(4):
+        assert np.array_equal(to_np(snaps[i]), want[i]), i
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        sequence()
+    for rep in (1, 2):
+        graph.replay()
+        torch.cuda.synchronize()
+        for i in range(4):
+            assert np.array_equal(to_np(snaps[i]), want[4 * rep + i]), (rep, i)
+    assert np.array_equal(to_np(theta.t), th_o) and np.array_equal(to_np(v.t), v_o)
+
+
 def test_host_gradient_entry_point():
     K, n = 4, 70_001
     theta, v, grads, _ = _make(K, n, "bf16", 11)
