@@ -401,6 +401,9 @@ def main():
                     help="how the sharded leg returns the updated ranges: one NCCL all-gather per tensor (one "
                          "rank per GPU), or device copies out of the peers' IPC-mapped buffers with gloo for the "
                          "host-side protocol (also works with several ranks on one GPU)")
+    ap.add_argument("--ksweep-points", default="",
+                    help="with --extras ksweep: only these points, e.g. `f32:32,bf16:16` (default: the whole sweep)")
+    ap.add_argument("--ksweep-params", type=int, default=25_557_032, help="with --extras ksweep: parameters per point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -486,7 +489,8 @@ def main():
     extras = {}
     if rank == 0 and world == 1 and not args.no_extras and args.extras != "none":
         if args.extras == "ksweep":
-            extras = run_k_sweep(torch, B, peak)
+            pts = [(a, int(k)) for a, k in (x.split(":") for x in args.ksweep_points.split(",") if x)]
+            extras = run_k_sweep(torch, B, peak, P=args.ksweep_params, points=pts or None)
         else:
             extras = run_extras(torch, W, B, peak, job, only_asp=args.extras == "asp",
                                 with_cpu=not args.no_cpu_baseline)
@@ -632,7 +636,7 @@ def run_sharded(torch, W, B, ranks, peak, steps, how):
                     "unlike `value`, which counts independent replicas"}
 
 
-def run_k_sweep(torch, B, peak, P=25_557_032, steps=200):
+def run_k_sweep(torch, B, peak, P=25_557_032, steps=200, points=None):
     """The synchronous step on one flat bucket of P parameters for a range of worker counts and both
     gradient types (fixed batches, momentum 0.9): algorithmic GB/s against the measured copy peak."""
     out = {}
@@ -640,9 +644,12 @@ def run_k_sweep(torch, B, peak, P=25_557_032, steps=200):
     gen = torch.Generator(device=dev).manual_seed(0x0517)
     theta = torch.empty(P, device=dev).normal_(0, 0.05, generator=gen)
     v = torch.zeros(P, device=dev)
+    scrub = torch.empty(SCRUB_BYTES, dtype=torch.uint8, device=dev)
     for kind, gdt, esz in (("f32", torch.float32, 4), ("bf16", torch.bfloat16, 2)):
         grads = []
         for K in (1, 2, 4, 8, 12, 16, 20, 24, 32):
+            if points is not None and (kind, K) not in points:
+                continue
             while len(grads) < K:
                 grads.append(torch.empty(P, device=dev).normal_(0, 1e-3, generator=gen).to(gdt))
             o = B.Omni(K, 32 * K, 4, 96, 0.10)
@@ -661,9 +668,22 @@ def run_k_sweep(torch, B, peak, P=25_557_032, steps=200):
             bpp = esz * K + 16
             gbs = bpp * P / (ms * 1e-3) / 1e9
             grid, block = o.query_launch(K, B.BF16 if kind == "bf16" else B.F32)
+            # the same step timed alone after 512 MB were written through L2 (median of 30)
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(30)]
+            for a, c in ev:
+                scrub.fill_(1)
+                a.record()
+                o.aggregate_bsp(bs, b, 0.1, 0.9)
+                c.record()
+            torch.cuda.synchronize()
+            ms_cold = statistics.median(a.elapsed_time(c) for a, c in ev)
+            gbs_cold = bpp * P / (ms_cold * 1e-3) / 1e9
             out[f"{kind}_K{K}"] = {"ms_per_step": ms, "bytes_per_param": bpp, "achieved_gbs": gbs,
                                    "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-                                   "params_per_s": P / (ms * 1e-3), "grid": grid, "block": block}
+                                   "params_per_s": P / (ms * 1e-3), "grid": grid, "block": block,
+                                   "cold_l2": {"ms_per_step": ms_cold, "achieved_gbs": gbs_cold,
+                                               "frac_of_measured": gbs_cold / peak,
+                                               "frac_of_nominal_8TBs": gbs_cold / NOMINAL_HBM_GBS}}
             del o, bs
         del grads
         torch.cuda.empty_cache()

@@ -26,7 +26,8 @@
  * brute force on tiny inputs and a library optimiser; see tests/test_oracle_*.py.
  * Parity unpinned against the paper: the paper prints no controller trace and no aggregated
  * tensor, so the steps it leaves open -- rounding to integers, the order dead-band / bounds /
- * global-batch rule, Eq. 8 next to the bounds (oracle_rebatch, oracle_asp_report,
+ * global-batch rule, Eq. 8 next to the bounds, and the multiplicative variant of that rule behind
+ * ORACLE_FLAG_CONSERVE_MULTIPLICATIVE (oracle_rebatch, oracle_asp_report,
  * oracle_rebatch_static from the rounding step on) -- are pinned to this file's stated readings
  * through hand-derived cases, an exhaustive-search restatement of Eq. 8 and invariants, not to
  * numbers of the paper.  The element-wise rules (oracle_bsp_step_*, oracle_asp_apply_*,

@@ -163,6 +163,23 @@ template <typename G, int K> KernelInfo devlam_info()
             (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_smem_bytes<G>(K), true};
 }
 
+template <typename G, int K> KernelInfo devlam_short_info()
+{
+    constexpr TmaShape sh = tma_short_shape<G>(K);
+    return {reinterpret_cast<KernelFn>(&bsp_tma_kernel<G, K, sh.tile, sh.stages, sh.consumer_warps, false, true>),
+            (sh.consumer_warps + 1) * 32, 1, (unsigned long long)sh.tile, tma_ring_bytes(sh, K, int(sizeof(G))), true};
+}
+
+template <typename G> KernelInfo devlam_short_for(int K)
+{
+    switch (K) {
+#define OMNI_CASE(k) case k: return devlam_short_info<G, k>();
+        OMNI_FOR_EACH_K(OMNI_CASE)
+#undef OMNI_CASE
+    }
+    return {};
+}
+
 template <typename G> KernelInfo devlam_for(int K)
 {
     switch (K) {
@@ -178,6 +195,11 @@ template <typename G> KernelInfo devlam_for(int K)
 KernelInfo bulk_devlam_kernel(int dtype, int K)
 {
     return dtype == OMNI_BF16 ? devlam_for<__nv_bfloat16>(K) : devlam_for<float>(K);
+}
+
+KernelInfo bulk_devlam_short_kernel(int dtype, int K)
+{
+    return dtype == OMNI_BF16 ? devlam_short_for<__nv_bfloat16>(K) : devlam_short_for<float>(K);
 }
 
 int launch_device_rebatch(DeviceCtl *ctl, const omni_config &cfg, const double *measured_dev, int32_t *new_b_dev,

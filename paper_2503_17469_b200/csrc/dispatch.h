@@ -47,6 +47,7 @@ int short_launch_tiles_per_cta();
 // The synchronous ring kernel that reads its K weights from device memory (BspParams::lam_dev),
 // where the device-side controller leaves them (device_controller.cu).
 KernelInfo bulk_devlam_kernel(int dtype, int K);
+KernelInfo bulk_devlam_short_kernel(int dtype, int K);   // the same in the short-launch shape
 // The ring kernel as push with overwrite (Algorithm 2): one gradient stream, the snapshot in
 // place of theta (BspParams::src), optional copy of the result back to the snapshot (::copy).
 KernelInfo bulk_overwrite_kernel(int dtype);

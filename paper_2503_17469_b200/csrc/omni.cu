@@ -35,6 +35,7 @@ struct omni_ctx {
     omni::LaunchShape bulk_short_shape[2][OMNI_MAX_K + 1];  // [dtype][K], the same in its shape for short launches
     omni::LaunchShape bulk_seq_shape[2][OMNI_MAX_ASP_BATCH + 1];  // [dtype][M]
     omni::LaunchShape bulk_devlam_shape[2][OMNI_MAX_K + 1];       // [dtype][K], ring kernel with device-resident weights
+    omni::LaunchShape bulk_devlam_short_shape[2][OMNI_MAX_K + 1]; // [dtype][K], the same in the short-launch shape
     omni::LaunchShape asp_shape[2][2][2];               // [dtype][wide][momentum]
     omni::LaunchShape overwrite_shape[2][2];            // [dtype][wide]
     omni::LaunchShape bulk_overwrite_shape[2];          // [dtype], ring kernel as push with overwrite
@@ -213,10 +214,10 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
     LaunchShape *shape_slot = lam_dev ? &ctx->bulk_devlam_shape[dtype][K]
                               : bulk  ? &ctx->bulk_shape[dtype][K]
                                       : &ctx->bsp_shape[dtype][wide][K];
-    if (bulk && !lam_dev) {
+    if (bulk) {
         // a launch of a few rounds per CTA takes the short-launch shape, as long as that still
         // gives every SM a tile
-        const KernelInfo ks = bulk_short_kernel(dtype, K);
+        const KernelInfo ks = lam_dev ? bulk_devlam_short_kernel(dtype, K) : bulk_short_kernel(dtype, K);
         unsigned long long regular_tiles = 0, short_tiles = 0;
         for (int i = 0; i < n_buckets; ++i) {
             regular_tiles += (buckets[i].n + ki.tile - 1) / ki.tile;
@@ -225,7 +226,7 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
         const unsigned long long sms = (unsigned long long)ctx->sm_count;
         if (ks.fn != ki.fn && regular_tiles <= (unsigned long long)short_launch_tiles_per_cta() * sms && short_tiles >= sms) {
             ki = ks;
-            shape_slot = &ctx->bulk_short_shape[dtype][K];
+            shape_slot = lam_dev ? &ctx->bulk_devlam_short_shape[dtype][K] : &ctx->bulk_short_shape[dtype][K];
         }
     }
     LaunchShape &shape = *shape_slot;

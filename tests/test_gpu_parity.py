@@ -234,6 +234,29 @@ def test_results_are_deterministic():
     assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
 
 
+def test_two_contexts_on_two_streams_at_once():
+    """Two models stepped concurrently, each through its own context on its own stream (each
+    context has its own workspace, so the launches may overlap on the GPU): both end up with the
+    oracle's bits and their own squared norms."""
+    jobs = []
+    for j, (K, n, kind) in enumerate([(4, 700_001, "f32"), (16, 300_007, "bf16")]):
+        theta, v, grads, _ = _make(K, n, kind, 900 + j)
+        o = B.Omni(K, 32 * K, 1, 32 * K, 0.1)
+        bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+        jobs.append(dict(o=o, bs=bs, theta=theta, v=v, b=_random_batches(K, 32, 70 + j), stream=torch.cuda.Stream(),
+                         th_o=to_np(theta.t), v_o=to_np(v.t), g_np=[to_np(g.t) for g in grads]))
+    torch.cuda.synchronize()
+    for step in range(6):
+        for jb in jobs:                                   # interleaved enqueues, no synchronisation in between
+            jb["o"].aggregate_bsp(jb["bs"], jb["b"], 0.1, 0.9, 1e-4, stream=jb["stream"])
+    for jb in jobs:
+        jb["stream"].synchronize()
+        for step in range(6):
+            sq_o = O.bsp_step_f32(jb["g_np"], jb["b"], jb["th_o"], jb["v_o"], 0.1, 0.9, 1e-4)
+        assert np.array_equal(to_np(jb["theta"].t), jb["th_o"]) and np.array_equal(to_np(jb["v"].t), jb["v_o"])
+        assert abs(jb["o"].stats(stream=jb["stream"]).grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o
+
+
 def test_steps_replayed_from_a_cuda_graph():
     """Ten steps captured once into a CUDA graph (after one eager call, which binds the context
     to the device and sizes its launches) and replayed twice: the same bits as thirty eager
