@@ -6,9 +6,9 @@
 
 One step = one pass of the synchronous hot path on the ResNet-50-shaped mixed-precision
 workload (K=16 workers, 25.6M parameters, bfloat16 gradients, float32 master parameters and
-momentum, 25 MiB buckets): a controller re-batch from freshly jittered throughputs (host), the
-batch-size weights, the fused K-way weighted sum + momentum update + squared norm (one kernel
-launch over all buckets).  The asynchronous arrival path and the other configurations are timed
+momentum, 25 MiB buckets) through the one-call entry point omni_step_bsp: the batch-size
+weights, the fused K-way weighted sum + momentum update + squared-norm partials (one kernel
+launch over all buckets), and the controller's re-batch from freshly jittered throughputs (host).  The asynchronous arrival path and the other configurations are timed
 in the same run and reported under "extras".  Prints ONE JSON line on rank 0.
 
 Multi-GPU: the path has no exchange step, so N GPUs run N independent replicas; the value is
@@ -161,10 +161,12 @@ class BspJob:
         self.W = W
 
     def run(self, steps, schedule):
+        """``steps`` iterations of Algorithm 1 through the one-call entry point: fused aggregate +
+        update with the current batches, then the controller's re-batch from this iteration's
+        measurements."""
         o, bs, cfg = self.omni, self.buckets, self.cfg
         for i in range(steps):
-            b, _ = o.rebatch(schedule[i % len(schedule)])
-            o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+            o.step_bsp(bs, schedule[i % len(schedule)], cfg.lr, cfg.momentum, cfg.weight_decay)
 
     def timed(self, steps, warmup, schedule, sampler=None, barrier=None, repeats=REPEATS, reduce=None):
         """``warmup`` untimed steps, then ``repeats`` timed regions of exactly ``steps`` steps, each
@@ -203,15 +205,13 @@ class BspJob:
         o, bs, cfg = self.omni, self.buckets, self.cfg
         for i in range(3):
             between()
-            b, _ = o.rebatch(schedule[i % len(schedule)])
-            o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+            o.step_bsp(bs, schedule[i % len(schedule)], cfg.lr, cfg.momentum, cfg.weight_decay)
         torch.cuda.synchronize()
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         for i in range(steps):
             between()
-            b, _ = o.rebatch(schedule[i % len(schedule)])
             ev[i][0].record()
-            o.aggregate_bsp(bs, b, cfg.lr, cfg.momentum, cfg.weight_decay)
+            o.step_bsp(bs, schedule[i % len(schedule)], cfg.lr, cfg.momentum, cfg.weight_decay)
             ev[i][1].record()
         torch.cuda.synchronize()
         return [a.elapsed_time(c) for a, c in ev]

@@ -185,6 +185,20 @@ int omni_rebatch_static(omni_ctx *ctx, const double *capacity, int32_t *new_b);
 int omni_aggregate_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                        const int32_t *b, float lr, float momentum, float weight_decay, void *stream);
 
+/* One iteration of Algorithm 1's training loop in a single call: the aggregate + update of
+ * omni_aggregate_bsp with the controller's CURRENT batches (the ones the workers computed these
+ * gradients with: lambda_k = b_k / B), followed by omni_rebatch from `measured` (host, K values
+ * observed during this iteration), whose result applies to the next iteration's gradients.
+ * next_b[K] (host, out) receives the new batches, changed[K] (host, out, may be NULL) the 0/1 flags.
+ * Same arithmetic and the same kernels as the two calls made one after the other; it exists so
+ * that a step costs one trip through the binding instead of two, which matters for models small
+ * enough to be bound by the host's launch rate.  All arguments, the measurements included, are
+ * validated before the kernel is enqueued or the controller changes.
+ * Errors: those of omni_aggregate_bsp and omni_rebatch. */
+int omni_step_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                  const double *measured, float lr, float momentum, float weight_decay, int32_t *next_b,
+                  int32_t *changed, void *stream);
+
 /* One asynchronous arrival: worker `worker`'s gradient (buckets[i].grads[worker]), computed on
  * b_used samples, is applied to the server parameters with eta_k = float(lr * b_used / B)
  * (Eq. 5b; eta_k = lr with OMNI_ASP_NO_LR_SCALE):

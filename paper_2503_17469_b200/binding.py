@@ -31,7 +31,7 @@ EXPORTS = (
     "omni_apply_asp", "omni_aggregate_bsp_host", "omni_get_stats", "omni_last_cuda_error",
     "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
     "omni_ctl_to_device", "omni_ctl_from_device", "omni_rebatch_device", "omni_aggregate_bsp_device_batches",
-    "omni_shard_range", "omni_asp_push_pull", "omni_ctl_export", "omni_ctl_import",
+    "omni_shard_range", "omni_asp_push_pull", "omni_ctl_export", "omni_ctl_import", "omni_step_bsp",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
     L.omni_asp_report.argtypes = [vp, i32, i32, C.c_double, C.POINTER(i32)]
     L.omni_rebatch_static.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i32)]
     L.omni_aggregate_bsp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(i32), f32, f32, f32, vp]
+    L.omni_step_bsp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, C.POINTER(C.c_double), f32, f32, f32,
+                                C.POINTER(i32), C.POINTER(i32), vp]
     L.omni_apply_asp.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, i32, i32, f32, f32, f32, vp]
     L.omni_apply_asp_batch.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, i32, C.POINTER(i32), C.POINTER(i32),
                                        C.POINTER(i32), f32, f32, f32, vp]
@@ -286,6 +288,16 @@ class Omni:
                       weight_decay: float = 0.0, stream=None) -> None:
         self._check(lib().omni_aggregate_bsp(self._h, buckets.array, buckets.n_buckets, buckets.dtype,
                                              self._i32K(*b), lr, momentum, weight_decay, self._stream(stream)))
+
+    def step_bsp(self, buckets: BucketSet, measured: Sequence[float], lr: float, momentum: float = 0.0,
+                 weight_decay: float = 0.0, stream=None) -> List[int]:
+        """One iteration of Algorithm 1 in one call: aggregate + update with the current batches,
+        then re-batch from ``measured``; returns the batches for the next iteration."""
+        nb = self._i32K()
+        self._check(lib().omni_step_bsp(self._h, buckets.array, buckets.n_buckets, buckets.dtype,
+                                        self._f64K(*measured), lr, momentum, weight_decay, nb, None,
+                                        self._stream(stream)))
+        return list(nb)
 
     def aggregate_bsp_host(self, buckets: BucketSet, host_grads: Sequence[Sequence], b: Sequence[int], lr: float,
                            momentum: float = 0.0, weight_decay: float = 0.0, stream=None) -> float:

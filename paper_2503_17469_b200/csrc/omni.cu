@@ -477,6 +477,39 @@ int omni_aggregate_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buck
     return OMNI_OK;
 }
 
+int omni_step_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
+                  const double *measured, float lr, float momentum, float weight_decay, int32_t *next_b,
+                  int32_t *changed, void *stream)
+{
+    if (!ctx || !measured || !next_b) return OMNI_ERR_NULL;
+    int rc = check_buckets(ctx, buckets, n_buckets, grad_dtype, -1, momentum);
+    if (rc != OMNI_OK) return rc;
+    // the weights of this step come from the batches the gradients were computed with
+    int32_t used[OMNI_MAX_K];
+    std::memcpy(used, ctx->ctl.batches(), sizeof(int32_t) * ctx->ctl.K());
+    // Re-batch first: it is host arithmetic, and a refused measurement leaves the controller as it
+    // was, so nothing has been enqueued yet if it fails.  Keep what is needed to undo it should
+    // the launch fail afterwards.
+    int32_t old_b[OMNI_MAX_K], old_seen[OMNI_MAX_K];
+    double old_t[OMNI_MAX_K];
+    ctx->ctl.export_state(old_b, old_t, old_seen);
+    rc = ctx->ctl.rebatch(measured, next_b, changed);
+    if (rc != OMNI_OK) return rc;
+    float lam[OMNI_MAX_K];
+    const double wsum = fill_weights(ctx, used, lam);
+    rc = ensure_device(ctx);
+    if (rc == OMNI_OK)
+        rc = enqueue_bsp(ctx, buckets, n_buckets, grad_dtype, lam, nullptr, lr, momentum, weight_decay,
+                         static_cast<cudaStream_t>(stream));
+    if (rc != OMNI_OK) {
+        ctx->ctl.import_state(old_b, old_t, old_seen);   // undo the re-batch
+        return rc;
+    }
+    ctx->tally.weight_sum = wsum;
+    ctx->tally.steps += 1;
+    return OMNI_OK;
+}
+
 int omni_aggregate_bsp_host(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                             const void *const *host_grads, const int32_t *b, float lr, float momentum,
                             float weight_decay, void *stream, double *grad_sqnorm)

@@ -234,6 +234,38 @@ def test_results_are_deterministic():
     assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
 
 
+@pytest.mark.parametrize("kind", ["f32", "bf16"])
+def test_one_call_step_is_aggregate_then_rebatch(kind):
+    """omni_step_bsp over twelve iterations with jittered throughputs: each iteration aggregates
+    with the batches of the previous re-batch (the ones the gradients were computed with), then
+    re-batches; parameters, momentum, norms and batches equal the oracle's and the two-call
+    sequence's."""
+    K, n = 8, 3 * 8192 + 29
+    theta, v, grads, _ = _make(K, n, kind, 1234)
+    o = B.Omni(K, 256, 4, 96, 0.1)
+    two = B.Omni(K, 256, 4, 96, 0.1)
+    ora = O.Controller(K, 256, 4, 96, 0.1)
+    bs = B.BucketSet([theta.t], [[g.t for g in grads]], [v.t])
+    th2, v2 = theta.t.clone(), v.t.clone()
+    bs2 = B.BucketSet([th2], [[g.t for g in grads]], [v2])
+    th_o, v_o, g_np = to_np(theta.t), to_np(v.t), [to_np(g.t) for g in grads]
+    rng = np.random.default_rng(3)
+    base = 8.0 ** rng.random(K)
+    for it in range(12):
+        T = base * (1.0 + 0.2 * (2.0 * rng.random(K) - 1.0))
+        used = ora.batches.copy()
+        nxt = o.step_bsp(bs, T.tolist(), 0.1, 0.9, 1e-4)
+        two.aggregate_bsp(bs2, two.batches, 0.1, 0.9, 1e-4)
+        nxt2, _ = two.rebatch(T.tolist())
+        sq_o = O.bsp_step_f32(g_np, used, th_o, v_o, 0.1, 0.9, 1e-4)
+        want, _ = ora.rebatch(T)
+        assert nxt == nxt2 == want.tolist() == o.batches
+        st = o.stats()
+        assert abs(st.grad_sqnorm - sq_o) <= SQNORM_RTOL * sq_o and st.steps == it + 1
+    assert np.array_equal(to_np(theta.t), th_o) and np.array_equal(to_np(v.t), v_o)
+    assert np.array_equal(to_np(th2), th_o) and np.array_equal(to_np(v2), v_o)
+
+
 def test_two_contexts_on_two_streams_at_once():
     """Two models stepped concurrently, each through its own context on its own stream (each
     context has its own workspace, so the launches may overlap on the GPU): both end up with the

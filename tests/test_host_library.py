@@ -196,6 +196,16 @@ def test_argument_validation_happens_before_any_cuda_call():
     assert asp(2, 32, 0, 0.1, 0.0, 0.0, None) == B.ERR_BAD_WORKER
     assert asp(0, 0, 0, 0.1, 0.0, 0.0, None) == B.ERR_BAD_BATCH
     assert asp(0, 32, -1, 0.1, 0.0, 0.0, None) == B.ERR_BAD_TAU
+    # the one-call step: the measurements are validated before anything is enqueued, and a call that
+    # fails afterwards (here: no usable device memory behind the made-up pointers is never reached,
+    # the measurement is refused first) leaves the controller as it was
+    nb = (C.c_int32 * 2)()
+    step = lambda m, *a: L.omni_step_bsp(o._h, bk, 1, 0, m, 0.1, 0.9, 0.0, *a)
+    assert step(None, nb, None, None) == B.ERR_NULL
+    assert step((C.c_double * 2)(1.0, 2.0), None, None, None) == B.ERR_NULL
+    assert step((C.c_double * 2)(1.0, 0.0), nb, None, None) == B.ERR_BAD_MEASUREMENT
+    assert step((C.c_double * 2)(float("nan"), 1.0), nb, None, None) == B.ERR_BAD_MEASUREMENT
+    assert o.batches == [32, 32]
     # the device-resident controller: nothing works before the device copy exists
     assert L.omni_ctl_to_device(None, None) == B.ERR_NULL
     assert L.omni_ctl_from_device(None, None) == B.ERR_NULL
