@@ -852,7 +852,8 @@ def run_extras(torch, W, B, peak, headline_job, only_asp=False, with_cpu=True):
     st = o.stats()
     out["resnet50_asp"] = asp_line(times, cfg.steps, cfg.bytes_per_param(), "asp_tma_f32_single_arrival")
     out["resnet50_asp"].update({"launches_per_arrival": (o.kernel_launches - l0) / (REPEATS * cfg.steps),
-                                "tau_max": st.tau_max, "tau_hist_0_31_overflow": st.tau_hist})
+                                "tau_max": st.tau_max, "tau_mean": st.tau_mean,
+                                "tau_hist_0_31_overflow": st.tau_hist})
     # one arrival when theta is not in L2: 512 MB written between two arrivals, each timed on its own
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(40)]
     i_next = 50 + REPEATS * cfg.steps

@@ -117,8 +117,9 @@ typedef struct {
     double weight_sum;   /* sum_k lambda_k (as rounded to float) of that call */
     uint64_t steps;      /* synchronous steps enqueued */
     uint64_t arrivals;   /* asynchronous arrivals enqueued */
-    uint64_t tau_hist[OMNI_TAU_BINS];
+    uint64_t tau_hist[OMNI_TAU_BINS]; /* arrivals by staleness 0..31, last bin: 32 and more */
     int32_t tau_max;
+    uint64_t tau_sum;    /* sum of the staleness of all arrivals (mean = tau_sum / arrivals) */
 } omni_stats;
 
 typedef struct omni_ctx omni_ctx;
@@ -266,6 +267,11 @@ int omni_asp_push_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buck
  *   next omni_ctl_from_device returns (once).  The host controller is not touched: host calls
  *   (omni_rebatch, omni_get_batches, ...) keep seeing the state of the last
  *   omni_ctl_from_device.
+ * omni_asp_report_device: evalBsz of Algorithm 2 (omni_asp_report) on the device copy: worker and
+ *   b_used are host values, measured_dev = DEVICE double[1] (8-byte aligned), new_b_k_dev = DEVICE
+ *   int32[1] out or NULL.  Stores the worker's batch and smoothed time in the device copy and,
+ *   once every worker has an entry, re-evaluates all K entries (no Eq. 8); a bad measurement is
+ *   recorded as for omni_rebatch_device.  Same integers as omni_asp_report, bit for bit.
  * omni_aggregate_bsp_device_batches: omni_aggregate_bsp with the weights the device copy holds
  *   (no `b` argument; nothing is checked against B on the host).  Always the bulk-copy ring kernel.
  * omni_ctl_from_device: synchronises `stream`, copies the device copy back into the host
@@ -273,10 +279,13 @@ int omni_asp_push_pull(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buck
  * omni_ctl_to_device and omni_ctl_from_device copy between pageable host memory and the device and
  * are not meant to be captured; omni_rebatch_device and omni_aggregate_bsp_device_batches are
  * plain kernel launches.
- * Errors: NULL, BAD_CONFIG (no device copy yet; or as omni_aggregate_bsp), ALIGN, CUDA. */
+ * Errors: NULL, BAD_CONFIG (no device copy yet; or as omni_aggregate_bsp), ALIGN, CUDA;
+ * omni_asp_report_device also BAD_WORKER, BAD_BATCH. */
 int omni_ctl_to_device(omni_ctx *ctx, void *stream);
 int omni_ctl_from_device(omni_ctx *ctx, void *stream);
 int omni_rebatch_device(omni_ctx *ctx, const double *measured_dev, int32_t *new_b_dev, void *stream);
+int omni_asp_report_device(omni_ctx *ctx, int32_t worker, int32_t b_used, const double *measured_dev,
+                           int32_t *new_b_k_dev, void *stream);
 int omni_aggregate_bsp_device_batches(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, int32_t grad_dtype,
                                       float lr, float momentum, float weight_decay, void *stream);
 

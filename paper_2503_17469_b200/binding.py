@@ -32,6 +32,7 @@ EXPORTS = (
     "omni_query_launch", "omni_kernel_launches", "omni_aggregate_bsp_noalloc", "omni_apply_asp_batch", "omni_asp_pull", "omni_asp_push_overwrite", "omni_selftest_wait_expiry",
     "omni_ctl_to_device", "omni_ctl_from_device", "omni_rebatch_device", "omni_aggregate_bsp_device_batches",
     "omni_shard_range", "omni_asp_push_pull", "omni_ctl_export", "omni_ctl_import", "omni_step_bsp",
+    "omni_asp_report_device",
 )
 MAX_ASP_BATCH = 16
 NOALLOC_MAX_BUCKETS = 8
@@ -50,7 +51,8 @@ class omni_bucket(C.Structure):
 
 class omni_stats(C.Structure):
     _fields_ = [("grad_sqnorm", C.c_double), ("weight_sum", C.c_double), ("steps", C.c_uint64),
-                ("arrivals", C.c_uint64), ("tau_hist", C.c_uint64 * TAU_BINS), ("tau_max", C.c_int32)]
+                ("arrivals", C.c_uint64), ("tau_hist", C.c_uint64 * TAU_BINS), ("tau_max", C.c_int32),
+                ("tau_sum", C.c_uint64)]
 
 
 _lib: Optional[C.CDLL] = None
@@ -88,6 +90,7 @@ def lib() -> C.CDLL:
     L.omni_ctl_to_device.argtypes = [vp, vp]
     L.omni_ctl_from_device.argtypes = [vp, vp]
     L.omni_rebatch_device.argtypes = [vp, vp, vp, vp]
+    L.omni_asp_report_device.argtypes = [vp, i32, i32, vp, vp, vp]
     L.omni_aggregate_bsp_device_batches.argtypes = [vp, C.POINTER(omni_bucket), i32, i32, f32, f32, f32, vp]
     L.omni_shard_range.argtypes = [C.c_uint64, i32, i32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.omni_ctl_export.argtypes = [vp, vp, C.POINTER(C.c_uint64)]
@@ -138,6 +141,11 @@ class Stats:
     arrivals: int
     tau_hist: List[int]
     tau_max: int
+    tau_sum: int = 0
+
+    @property
+    def tau_mean(self) -> float:
+        return self.tau_sum / self.arrivals if self.arrivals else 0.0
 
 
 class BucketSet:
@@ -364,6 +372,15 @@ class Omni:
                                               C.c_void_p(new_b.data_ptr()) if new_b is not None else None,
                                               self._stream(stream)))
 
+    def asp_report_device(self, worker: int, b_used: int, measured, new_b=None, stream=None) -> None:
+        """evalBsz on the device copy: ``measured`` is a one-element float64 CUDA tensor, ``new_b`` an
+        optional one-element int32 CUDA tensor that receives the worker's new batch."""
+        assert measured.is_cuda and measured.element_size() == 8 and measured.numel() >= 1
+        assert new_b is None or (new_b.is_cuda and new_b.element_size() == 4 and new_b.numel() >= 1)
+        self._check(lib().omni_asp_report_device(self._h, worker, b_used, C.c_void_p(measured.data_ptr()),
+                                                 C.c_void_p(new_b.data_ptr()) if new_b is not None else None,
+                                                 self._stream(stream)))
+
     def aggregate_bsp_device_batches(self, buckets: BucketSet, lr: float, momentum: float = 0.0,
                                      weight_decay: float = 0.0, stream=None) -> None:
         self._check(lib().omni_aggregate_bsp_device_batches(self._h, buckets.array, buckets.n_buckets, buckets.dtype,
@@ -381,7 +398,7 @@ class Omni:
         s = omni_stats()
         st = C.c_void_p(0) if stream is None and not self._device_used() else self._stream(stream)
         self._check(lib().omni_get_stats(self._h, C.byref(s), st))
-        return Stats(s.grad_sqnorm, s.weight_sum, s.steps, s.arrivals, list(s.tau_hist), s.tau_max)
+        return Stats(s.grad_sqnorm, s.weight_sum, s.steps, s.arrivals, list(s.tau_hist), s.tau_max, s.tau_sum)
 
     def selftest_wait_expiry(self, stream=None) -> None:
         """Enqueue the diagnostic kernel whose bounded wait runs out (next ``stats()`` raises TIMEOUT)."""

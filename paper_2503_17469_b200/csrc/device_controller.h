@@ -22,6 +22,10 @@ struct DeviceCtl {
     uint32_t rebatches;          // device re-batches that completed
 };
 
+// Enqueues the one-warp asynchronous report kernel (evalBsz); returns the cudaError_t as int.
+int launch_device_report(DeviceCtl *ctl, const omni_config &cfg, int32_t worker, int32_t b_used, const double *measured_dev,
+                         int32_t *new_b_dev, void *stream);
+
 // Enqueues the one-warp re-batch kernel (device_controller.cu); returns the cudaError_t as int.
 int launch_device_rebatch(DeviceCtl *ctl, const omni_config &cfg, const double *measured_dev, int32_t *new_b_dev,
                           void *stream);

@@ -187,6 +187,16 @@ int finalize_sqnorm(omni_ctx *ctx, cudaStream_t stream)
     return OMNI_OK;
 }
 
+// Staleness bookkeeping of one asynchronous arrival (the paper defines no staleness-dependent
+// factor, so tau is only tallied): histogram with an overflow bin, maximum, sum.
+void tally_arrival(omni_ctx *ctx, int32_t tau)
+{
+    ctx->tally.arrivals += 1;
+    ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
+    if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+    ctx->tally.tau_sum += uint64_t(tau);
+}
+
 // Eq. 4b: lambda_k = b_k / sum b, evaluated in double and rounded once to float.
 double fill_weights(const omni_ctx *ctx, const int32_t *b, float *lam)
 {
@@ -568,9 +578,7 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
         rc = enqueue_seq(ctx, buckets, n_buckets, grad_dtype, 1, &worker, &b_used, lr, momentum, weight_decay,
                          static_cast<cudaStream_t>(stream));
         if (rc != OMNI_OK) return rc;
-        ctx->tally.arrivals += 1;
-        ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
-        if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+        tally_arrival(ctx, tau);
         return OMNI_OK;
     }
     const bool wide = all_aligned32(buckets, n_buckets, worker, worker + 1);
@@ -603,9 +611,7 @@ int omni_apply_asp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets,
         rc = launch(ctx, ki, grid, &p, static_cast<cudaStream_t>(stream));
         if (rc != OMNI_OK) return rc;
     }
-    ctx->tally.arrivals += 1;
-    ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
-    if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+    tally_arrival(ctx, tau);
     return OMNI_OK;
 }
 
@@ -631,9 +637,7 @@ int omni_apply_asp_batch(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_bu
                      static_cast<cudaStream_t>(stream));
     if (rc != OMNI_OK) return rc;
     for (int a = 0; a < m; ++a) {
-        ctx->tally.arrivals += 1;
-        ctx->tally.tau_hist[tau[a] < OMNI_TAU_BINS - 1 ? tau[a] : OMNI_TAU_BINS - 1] += 1;
-        if (tau[a] > ctx->tally.tau_max) ctx->tally.tau_max = tau[a];
+        tally_arrival(ctx, tau[a]);
     }
     return OMNI_OK;
 }
@@ -749,9 +753,7 @@ static int push_overwrite(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_b
                     OMNI_CUDA(ctx, cudaMemcpyAsync(snapshots[j], buckets[j].param, buckets[j].n * sizeof(float),
                                                    cudaMemcpyDeviceToDevice, s));
     }
-    ctx->tally.arrivals += 1;
-    ctx->tally.tau_hist[tau < OMNI_TAU_BINS - 1 ? tau : OMNI_TAU_BINS - 1] += 1;
-    if (tau > ctx->tally.tau_max) ctx->tally.tau_max = tau;
+    tally_arrival(ctx, tau);
     return OMNI_OK;
 }
 
@@ -816,6 +818,25 @@ int omni_rebatch_device(omni_ctx *ctx, const double *measured_dev, int32_t *new_
     int rc = ensure_device(ctx);
     if (rc != OMNI_OK) return rc;
     const int e = launch_device_rebatch(ctx->dctl, ctx->ctl.config(), measured_dev, new_b_dev, stream);
+    if (e != 0) {
+        ctx->last_cuda = e;
+        return OMNI_ERR_CUDA;
+    }
+    ctx->launches += 1;
+    return OMNI_OK;
+}
+
+int omni_asp_report_device(omni_ctx *ctx, int32_t worker, int32_t b_used, const double *measured_dev,
+                           int32_t *new_b_dev, void *stream)
+{
+    if (!ctx || !measured_dev) return OMNI_ERR_NULL;
+    if (worker < 0 || worker >= ctx->ctl.K()) return OMNI_ERR_BAD_WORKER;
+    if (b_used < 1) return OMNI_ERR_BAD_BATCH;
+    if (!ctx->dctl) return OMNI_ERR_BAD_CONFIG;
+    if ((reinterpret_cast<uintptr_t>(measured_dev) & 7u) || (reinterpret_cast<uintptr_t>(new_b_dev) & 3u)) return OMNI_ERR_ALIGN;
+    int rc = ensure_device(ctx);
+    if (rc != OMNI_OK) return rc;
+    const int e = launch_device_report(ctx->dctl, ctx->ctl.config(), worker, b_used, measured_dev, new_b_dev, stream);
     if (e != 0) {
         ctx->last_cuda = e;
         return OMNI_ERR_CUDA;

@@ -77,6 +77,62 @@ def test_device_rebatch_matches_the_oracle_bit_for_bit(seed):
     assert o.rebatch(list(m))[0] == [int(x) for x in ref.rebatch(m)[0]]
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_device_report_matches_the_oracle_bit_for_bit(seed):
+    """evalBsz on the device copy: 150 reports of randomly chosen workers (throughput or time
+    input, smoothing, now and then a batch that differs from the server's entry); after every
+    report the returned batch equals the oracle's, at the end the whole map does, and the host
+    controller continues from the downloaded state exactly as the oracle does."""
+    rng = np.random.default_rng(7000 + seed)
+    K = int(rng.integers(1, 33))
+    alpha = float(rng.choice([1.0, 0.5, 0.25]))
+    flags = int(rng.choice([0, B.INPUT_IS_TIME]))
+    o = B.Omni(K, 32 * K, 4, 96, 0.10, alpha, B.ASP, flags)
+    ref = O.Controller(K, 32 * K, 4, 96, 0.10, alpha, O.MODE_ASP, _oracle_flags(flags))
+    o.ctl_to_device()
+    T = 8.0 ** rng.random(K)
+    cur = [32] * K
+    measured = torch.empty(1, dtype=torch.float64, device=DEV)
+    out = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for ev in range(150):
+        k = int(rng.integers(0, K))
+        used = cur[k] if rng.random() < 0.8 else int(rng.integers(4, 97))
+        thr = float(T[k] * (1.0 + 0.1 * rng.uniform(-1, 1)))
+        m = used / thr if flags & B.INPUT_IS_TIME else thr
+        measured.fill_(m)
+        o.asp_report_device(k, used, measured, out)
+        want = ref.asp_report(k, used, m)
+        got = int(out.item())
+        assert got == want, (seed, ev, k, got, want)
+        cur[k] = got
+    assert o.ctl_from_device() == [int(x) for x in ref.batches]
+    k = int(rng.integers(0, K))
+    assert o.asp_report(k, cur[k], float(T[k])) == ref.asp_report(k, cur[k], float(T[k]))
+
+
+def test_device_report_hand_case_and_refused_measurement():
+    """The hand-derived report sequence R1 (a reported batch that differs from the server's entry,
+    alpha = 0.25, time input) on the device copy; a measurement that is not positive changes nothing
+    and is reported once."""
+    o = B.Omni(2, 64, 4, 96, 0.10, 0.25, B.ASP, B.INPUT_IS_TIME)
+    o.ctl_to_device()
+    m = torch.empty(1, dtype=torch.float64, device=DEV)
+    out = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for worker, used, t, ret, after in ((0, 32, 8.0, 32, [32, 32]), (1, 32, 4.0, 48, [24, 48]),
+                                        (0, 20, 6.0, 15, [15, 69]), (1, 69, 6.0, 92, [12, 92])):
+        m.fill_(t)
+        o.asp_report_device(worker, used, m, out)
+        assert int(out.item()) == ret
+        assert o.ctl_from_device() == after
+    m.fill_(0.0)
+    out.fill_(-7)
+    o.asp_report_device(0, 12, m, out)
+    with pytest.raises(B.OmniError) as e:
+        o.ctl_from_device()
+    assert e.value.status == B.ERR_BAD_MEASUREMENT and int(out.item()) == -7
+    assert o.ctl_from_device() == [12, 92]
+
+
 def test_device_rebatch_reproduces_the_hand_case():
     """Throughputs (1,2,4,8), B = 64, bounds (2,48), dead-band 10 %: (2,6,19,37), (6,9,17,32),
     (4,8,16,36), then steady -- the hand-derived trace the host controller is pinned to."""

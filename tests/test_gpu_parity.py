@@ -564,6 +564,7 @@ def test_asp_event_stream_with_controller_feedback():
     assert t_lib == t_ora
     st = o.stats()
     assert st.arrivals == 1000 and st.tau_hist == tally.hist.tolist() and st.tau_max == tally.tau_max
+    assert st.tau_sum == sum(tau for _, tau, _ in t_lib) and st.tau_mean == st.tau_sum / 1000
     assert o.batches == ora.batches.tolist()
     assert assert_close(to_np(buf.theta), th_o, "f32") == 1.0
 

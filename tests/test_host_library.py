@@ -212,6 +212,10 @@ def test_argument_validation_happens_before_any_cuda_call():
     assert L.omni_ctl_from_device(o._h, None) == B.ERR_BAD_CONFIG
     assert L.omni_rebatch_device(o._h, None, None, None) == B.ERR_NULL
     assert L.omni_rebatch_device(o._h, 0x1000, None, None) == B.ERR_BAD_CONFIG
+    assert L.omni_asp_report_device(o._h, 0, 32, None, None, None) == B.ERR_NULL
+    assert L.omni_asp_report_device(o._h, 2, 32, 0x1000, None, None) == B.ERR_BAD_WORKER
+    assert L.omni_asp_report_device(o._h, 0, 0, 0x1000, None, None) == B.ERR_BAD_BATCH
+    assert L.omni_asp_report_device(o._h, 0, 32, 0x1000, None, None) == B.ERR_BAD_CONFIG   # no device copy yet
     assert L.omni_aggregate_bsp_device_batches(None, bk, 1, 0, 0.1, 0.9, 0.0, None) == B.ERR_NULL
     assert L.omni_aggregate_bsp_device_batches(o._h, bk, 1, 0, 0.1, 0.9, 0.0, None) == B.ERR_BAD_CONFIG
     assert o.kernel_launches == 0
