@@ -509,7 +509,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(HEADLINE, 12.0, torch, W)
 
-    ring = block == 288
+    ring = block == 224                      # 6 consumer warps + the producer warp: the bulk-copy ring
     traffic = recorded_traffic("bsp_tma_bf16_k16" if ring else "bsp_fused_bf16_k16")
     per_launch_s = ms * 1e-3 / max(launches, 1)
     if rank == 0:
@@ -528,7 +528,7 @@ def main():
             "pct_of_nominal_8TBs": 100 * line_main["frac_of_nominal_8TBs"],
             "roofline": {"bound": "hbm", "achieved": line_main["achieved_gbs"], "peak": peak, "unit": "GB/s",
                          "frac": line_main["frac_of_measured"], "peak_source": f"of {peak_kind}",
-                         "kernel": "bsp_tma_kernel<bf16,16,tile 2048,2 stages>" if ring else "bsp_fused_kernel<bf16,16>",
+                         "kernel": "bsp_tma_kernel<bf16,16,tile 2048,2 stages,6 consumer warps>" if ring else "bsp_fused_kernel<bf16,16>",
                          "bytes_per_launch": bytes_per_step,
                          "note": "frac = algorithmic bytes over the mean launch time of back-to-back steps; there part "
                                  "of theta/v comes from L2 (left by the previous step), so DRAM traffic per launch is "

@@ -378,8 +378,9 @@ int omni_selftest_wait_expiry(omni_ctx *ctx, void *stream);
 int omni_last_cuda_error(const omni_ctx *ctx);
 
 /* Persistent-grid size and block size the synchronous kernel for this K and dtype is launched
- * with on the current device (32-byte aligned buffers assumed; block = 288 means the bulk-copy
- * ring: 8 consumer warps + 1 producer warp), and the number of kernels enqueued so far. */
+ * with on the current device for a launch of ordinary length (32-byte aligned buffers assumed;
+ * block = 224 means the bulk-copy ring: 6 consumer warps + 1 producer warp; very short launches
+ * may use a ring of 288 threads), and the number of kernels enqueued so far. */
 int omni_query_launch(omni_ctx *ctx, int32_t K, int32_t grad_dtype, int32_t *grid, int32_t *block);
 uint64_t omni_kernel_launches(const omni_ctx *ctx);
 

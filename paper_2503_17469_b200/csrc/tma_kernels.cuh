@@ -95,8 +95,15 @@ struct TmaShape { int tile, stages, consumer_warps; };
 // larger ring loses 1-4 %).  Where that rule leaves copies of 2 KB (float K > 18, bfloat16
 // K > 16), a tile of one and a half times the size -- 3 KB copies, two stages of up to 108 KB --
 // wins 2-4 % (float K = 24: 7.10 vs 6.95 TB/s, K = 32: 6.93 vs 6.68; bfloat16 K = 32: 6.85 vs
-// 6.63), while 4 KB copies in a 213 KB ring lose again (float K = 24: 6.88).  Eight consumer
-// warps: 4 were 1-3 % slower, 6-12 the same, 16 slower again on bf16.
+// 6.63), while 4 KB copies in a 213 KB ring lose again (float K = 24: 6.88).  Six consumer
+// warps.  Scan of 4 / 6 / 8 warps on 25.6 M parameters (us per step, back to back; cold = L2
+// flushed before every step): bfloat16 K = 8 106.6 / 106.3 / 109.1 (cold 122.9 / 122.9 / 124.9),
+// bfloat16 K = 16 167.0 / 167.1 / 168.2 (cold 185.3 / 184.4 / 187.3), bfloat16 K = 32 295.6 /
+// 291.1 / 293.7, bfloat16 K = 4 81.4 / 82.1 / 82.4, float K = 8 165.9 / 166.4 / 166.9, float
+// K = 24 402.3 / 399.2 / 400.0, float K = 1, 4, 16 within 0.5 %; four warps lose 2.7 % at float
+// K = 2 (83.3 / 81.3 / 81.1) and sixteen were slower on bfloat16.  Six is never behind eight by
+// more than 0.4 % and ahead by up to 2.6 %: fewer resident warps spinning on barriers under the
+// power cap.  (The short-launch shape below keeps eight: 4.41 us against 4.67 with six.)
 template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
 {
     const int per_elem = K * int(sizeof(G)) + 8;
@@ -109,7 +116,7 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
     if (sizeof(G) == 4 && tile == 1024 && stages * stage > 160 * 1024) stages = 2;
     if (stages < 2) stages = 2;
     if (stages > 8) stages = 8;
-    return {tile, stages, 8};
+    return {tile, stages, 6};
 }
 // Short launches.  A launch that gives every CTA only a handful of tiles never reaches the ring's
 // steady state: its time is a few rounds of "fill a stage, consume it", and what counts is how
@@ -130,7 +137,7 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_short_shape(int
 {
     const TmaShape s = tma_shape<G>(K);
     const int per_elem = K * int(sizeof(G)) + 8;
-    if (s.tile < 4096 && 2 * (2 * s.tile) * per_elem <= 200 * 1024) return {2 * s.tile, 2, s.consumer_warps};
+    if (s.tile < 4096 && 2 * (2 * s.tile) * per_elem <= 200 * 1024) return {2 * s.tile, 2, 8};
     return s;
 }
 
@@ -148,7 +155,9 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_seq_shape(int M
     } else if (M == 1) {
         return {4096, 4, 16};
     }
-    return tma_shape<G>(M);
+    TmaShape s = tma_shape<G>(M);
+    s.consumer_warps = 8;   // the queues were tuned with eight
+    return s;
 }
 __host__ __device__ constexpr unsigned tma_ring_bytes(TmaShape s, int streams, int gsize)
 {

@@ -636,7 +636,7 @@ def test_resnet50_bf16_config_full_size():
     """The headline configuration at full size, 3 steps with the low-precision copy."""
     o = _bsp_config_run("resnet50_bf16", 3, lp=True)
     grid, block = o.query_launch(16, B.BF16)
-    assert grid % torch.cuda.get_device_properties(0).multi_processor_count == 0 and block in (288, 192, 256)
+    assert grid % torch.cuda.get_device_properties(0).multi_processor_count == 0 and block in (224, 192, 256)
 
 
 def test_resnet50_f32_config_full_size():
