@@ -80,8 +80,8 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
  * wait for the previous launch themselves, after their set-up).  The two flags force
  * one family; results are the same bit for bit.  A bounded wait of the ring that runs out
  * surfaces as OMNI_ERR_TIMEOUT from omni_get_stats.
- * Contract for the caller's own kernels on the same stream: the ring kernels (and the device
- * re-batch kernel) signal "dependents may launch" (griddepcontrol.launch_dependents) as soon as
+ * Contract for the caller's own kernels on the same stream: the ring kernels (and the one-warp
+ * kernels of the device-resident controller) signal "dependents may launch" (griddepcontrol.launch_dependents) as soon as
  * their set-up is done, long before their last store.  A kernel enqueued after a library call
  * in the ordinary way is not affected: the stream still runs it after the library's kernel has
  * finished.  A kernel that the caller launches WITH the programmatic-stream-serialization
@@ -91,6 +91,7 @@ typedef enum { OMNI_F32 = 0, OMNI_BF16 = 1 } omni_dtype;
  * launch only ordinary kernels and never signal early. */
 #define OMNI_BULK_COPY 8u
 #define OMNI_NO_BULK_COPY 16u
+/* omni_create refuses flag bits it does not know and both kernel-family flags together (BAD_CONFIG). */
 
 /* The "Input:" line of Algorithm 1 / Algorithm 2 (K, B, Delta b_k, b_min, b_max) plus the EWMA weight. */
 typedef struct {

@@ -19,6 +19,10 @@ int BatchController::validate(const omni_config &c)
     if (!(c.deadband >= 0.0) || !std::isfinite(c.deadband)) return OMNI_ERR_BAD_CONFIG;
     if (!(c.ewma_alpha > 0.0) || !(c.ewma_alpha <= 1.0)) return OMNI_ERR_BAD_CONFIG;
     if (c.mode != OMNI_BSP && c.mode != OMNI_ASP) return OMNI_ERR_BAD_CONFIG;
+    constexpr uint32_t known = OMNI_UNSCALED_MEAN | OMNI_ASP_NO_LR_SCALE | OMNI_INPUT_IS_TIME | OMNI_BULK_COPY |
+                               OMNI_NO_BULK_COPY | OMNI_CONSERVE_MULTIPLICATIVE;
+    if (c.flags & ~known) return OMNI_ERR_BAD_CONFIG;
+    if ((c.flags & OMNI_BULK_COPY) && (c.flags & OMNI_NO_BULK_COPY)) return OMNI_ERR_BAD_CONFIG;
     if (c.mode == OMNI_BSP) {
         const int64_t lo = int64_t(c.K) * c.b_min, hi = int64_t(c.K) * c.b_max;
         if (lo > c.global_batch || hi < c.global_batch) return OMNI_ERR_INFEASIBLE;

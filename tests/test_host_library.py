@@ -49,6 +49,8 @@ def test_create_validation():
     assert rc(deadband=-0.1) == B.ERR_BAD_CONFIG and rc(deadband=float("nan")) == B.ERR_BAD_CONFIG
     assert rc(ewma_alpha=0.0) == B.ERR_BAD_CONFIG and rc(ewma_alpha=1.5) == B.ERR_BAD_CONFIG
     assert rc(mode=7) == B.ERR_BAD_CONFIG
+    assert rc(flags=64) == B.ERR_BAD_CONFIG and rc(flags=B.BULK_COPY | B.NO_BULK_COPY) == B.ERR_BAD_CONFIG
+    assert rc(flags=B.UNSCALED_MEAN | B.INPUT_IS_TIME | B.CONSERVE_MULTIPLICATIVE | B.BULK_COPY) == B.OK
     assert B.lib().omni_create(None, None) == B.ERR_NULL
 
 
