@@ -137,6 +137,20 @@ def test_asp_report_hand_derived_sequences():
             assert o.batches == r["map_after"], case["name"]
 
 
+def test_library_batches_depend_only_on_throughput_ratios():
+    rng = np.random.default_rng(22)
+    for _ in range(50):
+        K = int(rng.integers(2, 33))
+        mult = bool(rng.uniform() < 0.5)
+        flags = B.CONSERVE_MULTIPLICATIVE if mult else 0
+        a = B.Omni(K, 32 * K, 4, 96, 0.1, 0.5, B.BSP, flags)
+        b = B.Omni(K, 32 * K, 4, 96, 0.1, 0.5, B.BSP, flags)
+        base = 8.0 ** rng.uniform(0, 1, K)
+        for step in range(5):
+            T = base * (1 + 0.2 * (2 * rng.uniform(0, 1, K) - 1))
+            assert a.rebatch(T.tolist())[0] == b.rebatch((T * 0.25).tolist())[0]
+
+
 def test_static_rebatch_matches_oracle():
     rng = np.random.default_rng(300)
     for _ in range(200):

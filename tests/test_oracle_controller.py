@@ -277,6 +277,25 @@ def test_equal_times_are_a_fixed_point_under_both_conservation_readings():
         assert c.rebatch([1, 2, 4, 9])[0].tolist() == [4, 8, 16, 36]
 
 
+def test_batches_depend_only_on_throughput_ratios():
+    """Eq. 6 in the form b* = T_k * mean_j(b_j / T_j): multiplying every throughput by the same
+    factor changes no batch.  With a power of two as the factor every intermediate scales exactly,
+    so the integers must be identical, synchronous and asynchronous, smoothed or not."""
+    rng = np.random.default_rng(21)
+    for _ in range(100):
+        K = int(rng.integers(2, 33))
+        mode = int(rng.integers(0, 2))
+        alpha = float(rng.choice([1.0, 0.5]))
+        a = O.Controller(K, 32 * K, 4, 96, 0.1, alpha, mode)
+        b = O.Controller(K, 32 * K, 4, 96, 0.1, alpha, mode)
+        base = 8.0 ** rng.uniform(0, 1, K)
+        for step in range(5):
+            T = base * (1 + 0.2 * (2 * rng.uniform(0, 1, K) - 1))
+            na, _ = a.rebatch(T)
+            nb, _ = b.rebatch(T * 64.0)
+            assert na.tolist() == nb.tolist()
+
+
 def test_errors_leave_state_untouched():
     c = O.Controller(4, 64, 2, 48, 0.1)
     before = c.batches.copy()
