@@ -143,13 +143,14 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_short_shape(int
 
 // The asynchronous apply of M queued arrivals uses the same geometry with M streams, except for
 // the shortest queues: with most of theta coming from L2 (see the alternating sweeps in omni.cu)
-// they are no longer DRAM-bound, and a deeper ring with sixteen consumer warps gains 2-6 %
-// (float M = 1: 8.20 vs 7.96 TB/s algorithmic; M = 2: 8.70 vs 8.24; M = 3: 8.55 vs 8.38;
-// bfloat16 M = 1: 8.73 vs 8.59; from M = 4 on nothing changed).
+// they are no longer DRAM-bound, and a deeper ring with more consumer warps gains 2-6 %
+// (float M = 1: 8.20 vs 7.96 TB/s algorithmic with sixteen warps, another 1.4 % with twelve;
+// M = 2: 8.70 vs 8.24; M = 3: 8.55 vs 8.38; bfloat16 M = 1: 8.73 vs 8.59, twelve warps 8.48;
+// from M = 4 on nothing changed, six warps or eight).
 template <typename G> __host__ __device__ constexpr TmaShape tma_seq_shape(int M)
 {
     if (sizeof(G) == 4) {
-        if (M == 1) return {4096, 4, 16};
+        if (M == 1) return {4096, 4, 12};   // 12 warps: 33.8 us per arrival; 16: 34.3; 10, 14: 36.6, 37.9; 8: 36.6
         if (M == 2) return {4096, 3, 16};
         if (M == 3) return {2048, 4, 16};
     } else if (M == 1) {
