@@ -41,7 +41,8 @@ KernelInfo bulk_kernel(int dtype, int K);
 KernelInfo bulk_seq_kernel(int dtype, int M);
 // The synchronous ring kernel in its shape for short launches (larger tiles, two stages; the same
 // kernel as bulk_kernel where no such shape fits), chosen when the regular shape would give a CTA
-// at most short_launch_tiles_per_cta() tiles and the larger tiles still number one per SM or more.
+// at most short_launch_tiles_per_cta() tiles (rounded up), the larger tiles exactly half as many,
+// and the larger tiles still number one per SM or more.
 KernelInfo bulk_short_kernel(int dtype, int K);
 int short_launch_tiles_per_cta();
 // The synchronous ring kernel that reads its K weights from device memory (BspParams::lam_dev),

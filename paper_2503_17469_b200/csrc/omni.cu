@@ -233,8 +233,11 @@ int enqueue_bsp(omni_ctx *ctx, const omni_bucket *buckets, int32_t n_buckets, in
             regular_tiles += (buckets[i].n + ki.tile - 1) / ki.tile;
             short_tiles += (buckets[i].n + ks.tile - 1) / ks.tile;
         }
+        // ... which pays when the larger tiles halve the number of fill-consume rounds exactly
         const unsigned long long sms = (unsigned long long)ctx->sm_count;
-        if (ks.fn != ki.fn && regular_tiles <= (unsigned long long)short_launch_tiles_per_cta() * sms && short_tiles >= sms) {
+        const unsigned long long rounds = (regular_tiles + sms - 1) / sms, short_rounds = (short_tiles + sms - 1) / sms;
+        if (ks.fn != ki.fn && short_tiles >= sms && rounds <= (unsigned long long)short_launch_tiles_per_cta() &&
+            2 * short_rounds == rounds) {
             ki = ks;
             shape_slot = lam_dev ? &ctx->bulk_devlam_short_shape[dtype][K] : &ctx->bulk_short_shape[dtype][K];
         }

@@ -126,12 +126,16 @@ template <typename G> __host__ __device__ constexpr TmaShape tma_shape(int K)
 // captured in a CUDA graph, 4096 x 2 runs a step in 4.40 us against 4.85 us for 2048 x 3 (and
 // 4.55 us for 2048 x 4, 5.2-5.4 us for 2048 x 2 and 1536 x 4; tiles of 1024 and 512 elements, which
 // balance the last wave better, were slower still: 8.0 and 11.4 us against 6.7 us before the norm's
-// final sum left the kernel).  The window is narrow: with 2^19 parameters (fewer large tiles than
-// SMs) the two shapes tie at 3.1 us, with 2^18 the regular one wins (2.4 vs 2.9 us), and from 2^21
-// parameters on (7 regular tiles per CTA) the regular shape's third stage wins again (6.7 vs
-// 7.1 us, 13.3 vs 13.7, 27.5 vs 28.4).  So the short shape is chosen when the regular shape
-// would give a CTA at most kShortLaunchTilesPerCta tiles and the large tiles still number at
-// least one per SM.
+// final sum left the kernel).  A short launch costs about a fixed part plus its number of
+// fill-consume rounds (tiles per CTA, rounded up) times a cost per round that is 1.6 times higher
+// for the large tiles, so the large tiles pay when they halve the number of rounds exactly and
+// lose when the regular count is odd: 2^19 parameters (2 regular rounds, fewer large tiles than
+// SMs) tie at 3.1 us, 2^18 (1 round) 2.4 vs 2.9 us, bfloat16 K = 8 on 3 * 2^18 parameters (3 rounds
+// against 2 large ones) 4.50 vs 4.79 us, on 2^20 (4 against 2) 5.25 vs 4.89 us (K = 7: 5.03 vs 4.73),
+// and from 2^21 parameters on (7 regular rounds) the regular shape's extra stage wins again (6.7 vs
+// 7.1 us, 13.3 vs 13.7, 27.5 vs 28.4).  So the short shape is chosen when the regular shape would
+// run at most kShortLaunchTilesPerCta rounds, the large tiles run exactly half as many, and they
+// still number at least one per SM.
 constexpr int kShortLaunchTilesPerCta = 4;
 template <typename G> __host__ __device__ constexpr TmaShape tma_short_shape(int K)
 {

@@ -123,12 +123,12 @@ def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
 @pytest.mark.parametrize("kind,K", [("f32", 4), ("bf16", 7), ("bf16", 8)])
 def test_short_launches_take_larger_tiles_with_the_same_bits(kind, K):
     """Launches of a few tiles per CTA run the ring in its short-launch shape (two stages of
-    4096-element tiles where they fit: float K = 4, bfloat16 K = 7 and 8).  Sizes inside that
-    window (a ragged tail, several buckets) and just outside it on both sides give the oracle's
-    bits either way."""
+    4096-element tiles where they fit: float K = 4, bfloat16 K = 7 and 8) when that halves the
+    number of rounds.  Sizes inside that window (four regular rounds: a ragged tail, several
+    buckets) and outside it (one, two, three and six rounds) give the oracle's bits either way."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     for sizes in ([sms * 4096 + 77], [sms * 2048 * 4 - 5], [sms * 2048 + 3], [5 * sms * 2048 + 4099],
-                  [300_001, 77, 450_003, 4096]):
+                  [300_001, 77, 450_003, 4096], [400_001, 77, 700_003, 4096]):
         bufs = [_make(K, n, kind, 4100 * K + n % 983, lp=True) for n in sizes]
         b = _random_batches(K, 32, K + sizes[0])
         o = B.Omni(K, 32 * K, 1, 32 * K, 0.1, flags=B.BULK_COPY)
