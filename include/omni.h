@@ -364,7 +364,9 @@ int omni_aggregate_bsp_noalloc(int32_t K, const omni_bucket *buckets, int32_t n_
                                const int32_t *b, uint32_t flags, float lr, float momentum, float weight_decay,
                                double *grad_sqnorm_dev, void *stream);
 
-/* Synchronises `stream` and fills *out (host). */
+/* Synchronises `stream` and fills *out (host).  The squared norm of the last synchronous step is
+ * summed here, by a one-warp kernel enqueued on `stream`: pass the stream that step was enqueued
+ * on, or one that has been ordered after it. */
 int omni_get_stats(omni_ctx *ctx, omni_stats *out, void *stream);
 
 /* Failure-path self-test (no counterpart in the paper).  Every device-side wait of the library is
